@@ -1,0 +1,215 @@
+/*
+ * muloco.h -- C ABI of the MuLoCo optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * One library call per line of the paper's Algorithm 1 that touches optimizer
+ * state: the inner step (Muon on hidden matrices, AdamW elsewhere) of K DiLoCo
+ * workers held as replicas on ONE GPU, and the outer synchronisation
+ * (pseudogradient, optional block quantisation, Nesterov outer SGD, broadcast).
+ * Gradients are supplied by the caller.
+ *
+ * Conventions
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer
+ *     to memory owned by the caller; the library never frees caller memory.
+ *     Arrays OF pointers (pointer tables) are always host arrays.
+ *   - The library owns only its workspace, its descriptor tables and the small
+ *     host state; muloco_destroy releases them.
+ *   - All matrices are row-major float32 unless stated; a vector is a 1 x n
+ *     matrix.
+ *   - Every call enqueues its work on the CUDA stream given at create time and
+ *     returns without waiting for the GPU.  Argument errors are reported by the
+ *     return value at once.  Conditions found on the device (non-finite
+ *     pseudogradient, a bounded wait that ran out) are written to a device
+ *     status word and reported by muloco_sync_status.  Nothing aborts or traps.
+ *   - Calls on one context are not thread-safe.
+ *   - There is no CPU fallback: without a CUDA device every compute call
+ *     returns MULOCO_ECUDA.
+ */
+#ifndef MULOCO_H
+#define MULOCO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MULOCO_API __attribute__((visibility("default")))
+#else
+#define MULOCO_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct muloco_ctx muloco_ctx; /* opaque */
+
+typedef enum {
+  MULOCO_OK = 0,
+  MULOCO_EINVAL = 1,     /* bad argument (NULL, out of range, J does not divide H ...) */
+  MULOCO_ESHAPE = 2,     /* unsupported shape */
+  MULOCO_ENOMEM = 3,     /* workspace allocation failed */
+  MULOCO_ECUDA = 4,      /* CUDA runtime/driver error, or no device */
+  MULOCO_ENONFINITE = 5, /* device saw a non-finite pseudogradient */
+  MULOCO_ETIMEOUT = 6,   /* a bounded wait inside a kernel ran out */
+  MULOCO_ESTATE = 7      /* call order / state blob mismatch */
+} muloco_status;
+
+typedef enum { MULOCO_MUON = 0, MULOCO_ADAMW = 1 } muloco_kind;
+typedef enum { MULOCO_NS_BF16 = 0, MULOCO_NS_FP32 = 1 } muloco_ns_mode;
+typedef enum { MULOCO_Q_NONE = 0, MULOCO_Q_INT4 = 4, MULOCO_Q_INT8 = 8 } muloco_quant;
+typedef enum { MULOCO_F32 = 0, MULOCO_BF16 = 1 } muloco_dtype;
+
+/* One parameter tensor of the model. */
+typedef struct {
+  int64_t rows, cols; /* a vector is rows = 1                                           */
+  int32_t kind;       /* muloco_kind: Muon for hidden matrices, AdamW for the rest
+                         (Section 5, "MuLoCo")                                          */
+  int32_t fragment;   /* 0..J-1: the subset synchronised together (Section 2,
+                         "Partitioned Communication")                                   */
+  float wd_mult;      /* multiplies the weight decay: 1 = decay, 0 = none (gains)       */
+  float lr_mult;      /* learning-rate multiplier; NaN selects the default:
+                         sqrt(cols/rows) for Muon (Section 5), 1 for AdamW              */
+} muloco_tensor_desc;
+
+typedef struct {
+  int32_t K, H, J;     /* workers, inner steps per round, fragments (J must divide H)   */
+  float muon_lr;       /* eta in W <- W - eta O - eta lambda W (Section 2, "Muon")      */
+  float muon_beta;     /* m <- beta m + g                                                */
+  float muon_wd;       /* lambda                                                         */
+  int32_t muon_nesterov; /* 1: orthogonalise g + beta m, 0: orthogonalise m            */
+  int32_t ns_steps;    /* Newton-Schulz iterations, 5 in the paper                       */
+  float ns_a, ns_b, ns_c; /* quintic coefficients, (3.4445, -4.7750, 2.0315)           */
+  float ns_eps;        /* X0 = U / (||U||_F + ns_eps)                                    */
+  int32_t ns_mode;     /* muloco_ns_mode                                                 */
+  int32_t wd_uses_scaled_lr; /* 1: the decay term uses the shape-rescaled eta too       */
+  float adam_lr, adam_beta1, adam_beta2, adam_eps, adam_wd; /* Section 4.3               */
+  int32_t adam_bias_correction; /* 1: divide by 1 - beta^t                              */
+  float outer_lr, outer_momentum; /* eta_out, mu of Eq. (3)                             */
+  int32_t quant;       /* muloco_quant: quantise -> dequantise the pseudogradient       */
+  int32_t quant_block; /* elements per absmax block along a row (128)                   */
+  int32_t grad_dtype;  /* muloco_dtype of the gradients given to muloco_inner_step      */
+  int32_t reserved;
+  uint64_t workspace_bytes; /* Newton-Schulz workspace budget; 0 lets the library pick  */
+} muloco_config;
+
+/* State buffers.  Every field is a HOST array of DEVICE pointers.
+ * Per-worker tables have K * n_tensors entries, entry [k * n_tensors + i]. */
+typedef struct {
+  float* const* theta_k;  /* [K][n]  worker replicas theta_k                            */
+  float* const* theta_g;  /* [n]     global parameters theta                            */
+  float* const* outer_u;  /* [n]     outer momentum u                                   */
+  float* const* state1_k; /* [K][n]  Muon momentum m, or Adam first moment              */
+  float* const* state2_k; /* [K][n]  Adam second moment (ignored for Muon tensors)      */
+} muloco_buffers;
+
+/* Algorithm 1, line 2.  Validates the arguments, records the tensor table,
+ * allocates the workspace (the only allocation the library makes), then
+ * enqueues u <- 0, inner state <- 0 and theta_k <- theta_g for every worker.
+ * `cuda_stream` is a cudaStream_t (NULL = the default stream).  n_tensors may
+ * be 0 for a context that only serves muloco_newton_schulz / muloco_quantize.
+ * On failure *out is NULL and the return value says why. */
+MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_tensor_desc* tensors,
+                            int32_t n_tensors, const muloco_buffers* bufs, void* cuda_stream,
+                            muloco_ctx** out);
+
+/* Releases workspace and tables (waits for the stream first). NULL is allowed. */
+MULOCO_API void muloco_destroy(muloco_ctx* ctx);
+
+/* Algorithm 1, lines 6-7 (Eq. 1) with the gradient given: one inner optimizer
+ * step for worker `worker` (0..K-1), or for all K workers batched when
+ * worker == -1.  `grads` is a host table of device pointers: [n_tensors] for one
+ * worker, [K][n_tensors] for all; each gradient has its tensor's shape and the
+ * dtype named by cfg.grad_dtype.  Gradients are read only.
+ * Hidden matrices (Section 2 "Muon", Section 5 "MuLoCo"):
+ *     m <- beta m + g;  U = g + beta m (Nesterov) or m;  O = NS_5(U / (||U||_F + eps));
+ *     W <- W - eta' O - eta' lambda W,  eta' = muon_lr * lr_scale * sqrt(cols/rows).
+ * Other tensors: AdamW (Section 4.3) with step size adam_lr * lr_scale.
+ * `lr_scale` is the learning-rate schedule's multiplier for this step. */
+MULOCO_API muloco_status muloco_inner_step(muloco_ctx* ctx, int32_t worker, const void* const* grads,
+                                float lr_scale);
+
+/* As muloco_inner_step, but `host_grads` is a host table of HOST pointers
+ * (pinned memory for full speed).  The gradients are copied to a device staging
+ * area owned by the library (allocated on first use) on the context's stream,
+ * then the step runs. */
+MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* ctx, int32_t worker,
+                                     const void* const* host_grads, float lr_scale);
+
+/* Algorithm 1, lines 9-13 (Eqs. 2-3) for the tensors of fragment `fragment`
+ * (0..J-1), or all tensors when fragment == -1, in one pass over memory:
+ *     Psi = (1/K) sum_k (theta_g - theta_k)   (fp32, k ascending, then * 1/K)
+ *     optional: Psi <- dequantise(quantise(Psi)) per block of quant_block elements
+ *               along a row (absmax scale, round to nearest even, int8 or int4)
+ *     u <- mu u + eta_out Psi;   theta_g <- theta_g - mu u - eta_out Psi
+ *     theta_k <- theta_g for every worker.
+ * Inner optimizer state is kept.  Syncing a fragment that is not due is allowed;
+ * the schedule is the caller's (see muloco_fragments_due). */
+MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* ctx, int32_t fragment);
+
+/* As muloco_outer_sync, then copies the new global parameters of every tensor
+ * of the fragment to host memory: host_theta_g is a host table [n_tensors] of
+ * HOST pointers (entries of tensors outside the fragment are not touched and
+ * may be NULL).  The copies are enqueued on the context's stream. */
+MULOCO_API muloco_status muloco_outer_sync_host(muloco_ctx* ctx, int32_t fragment, void* const* host_theta_g);
+
+/* Streaming schedule (Section 2, "Partitioned Communication"): fragment j
+ * (1-based) is due after inner step t > 0 when t mod H == (j H / J) mod H.
+ * Writes the 0-based due fragments to out_frags (host, room for J) and returns
+ * their count (0 if none, -1 on bad arguments). */
+MULOCO_API int32_t muloco_fragments_due(const muloco_ctx* ctx, int64_t step, int32_t* out_frags);
+
+/* Five-step quintic Newton-Schulz (Section 2, "Muon") on a batch of same-shape
+ * matrices, outside any optimizer state: X is [batch][rows][cols] (x_dtype),
+ * O has the same shape (o_dtype).  Each matrix is divided by its Frobenius norm
+ * (+ ns_eps) first; matrices with rows > cols are iterated on their transpose.
+ * ns_mode MULOCO_NS_BF16 runs the tensor-core engine (bf16 operands, fp32
+ * accumulation), MULOCO_NS_FP32 the fp32 engine.  X and O must not overlap. */
+MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* ctx, const void* X, int32_t x_dtype, void* O,
+                                   int32_t o_dtype, int32_t batch, int64_t rows, int64_t cols,
+                                   int32_t ns_mode);
+
+/* The block quantiser on its own (the benchmark's per-block absmax form of the
+ * linear quantisation of Section 2, "Compressed Communication"): psi is a
+ * rows x cols float32 matrix; writes, where non-NULL, one int8 code per element
+ * to `codes` (int4 codes are -7..7, unpacked), one float32 scale per block to
+ * `scales` ([rows][ceil(cols/block)]) and the dequantised values to `dequant`.
+ * bits is 8 or 4. */
+MULOCO_API muloco_status muloco_quantize(muloco_ctx* ctx, const float* psi, int64_t rows, int64_t cols,
+                              int32_t bits, int8_t* codes, float* scales, float* dequant);
+
+/* Test hook: the pseudogradient of tensor `tensor` (Eq. 2), exactly as
+ * muloco_outer_sync forms it, written to psi_out (float32, tensor's shape),
+ * without changing any state. */
+MULOCO_API muloco_status muloco_pseudogradient(muloco_ctx* ctx, int32_t tensor, float* psi_out);
+
+/* Small host state for checkpoint/resume: inner step counters per worker and
+ * sync counters per fragment.  Call with blob == NULL to get the size. */
+MULOCO_API muloco_status muloco_get_state(const muloco_ctx* ctx, void* host_blob, size_t* nbytes);
+MULOCO_API muloco_status muloco_set_state(muloco_ctx* ctx, const void* host_blob, size_t nbytes);
+
+/* Phase timers (CUDA events on the context's stream). */
+enum {
+  MULOCO_PH_PROLOGUE = 0, /* momentum + bf16/fp32 staging + norms                     */
+  MULOCO_PH_NS = 1,       /* Newton-Schulz GEMMs, including the fused final update    */
+  MULOCO_PH_ADAMW = 2,
+  MULOCO_PH_SYNC = 3,
+  MULOCO_PH_COPY = 4,     /* host<->device copies of the *_host calls                 */
+  MULOCO_N_PHASES = 5
+};
+MULOCO_API muloco_status muloco_set_timing(muloco_ctx* ctx, int32_t enabled);
+/* Waits for the stream, writes the milliseconds accumulated per phase since the
+ * last call to ms[MULOCO_N_PHASES] and the number of kernel launches since the
+ * last call to *launches (either may be NULL), then resets both. */
+MULOCO_API muloco_status muloco_get_timings(muloco_ctx* ctx, float* ms, int64_t* launches);
+
+/* Waits for the stream and returns the device status word as a muloco_status
+ * (MULOCO_OK, MULOCO_ENONFINITE, MULOCO_ETIMEOUT, MULOCO_ECUDA); clears it. */
+MULOCO_API muloco_status muloco_sync_status(muloco_ctx* ctx);
+
+/* Text of the last error on this context (or of the last failed create when
+ * ctx is NULL).  The string is owned by the library. */
+MULOCO_API const char* muloco_last_error(const muloco_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MULOCO_H */

@@ -1,0 +1,249 @@
+// HBM-bound elementwise kernels of the inner step:
+//   - Muon prologue: m <- beta m + g, NS input U staged as bf16/fp32 (transposed
+//     when the tensor has more rows than columns), partial sums of U^2 for the
+//     Frobenius norm (Section 2, "Muon").
+//   - scale finalisation: r = 1 / (||U||_F + eps) per matrix, deterministic order.
+//   - fused AdamW (Section 4.3) over a flat list of (worker, tensor) segments.
+#include "internal.h"
+
+namespace muloco {
+
+namespace {
+
+constexpr int PRO_TI = 32;    // tile rows of X (the s dimension)
+constexpr int PRO_TJ = 128;   // tile cols of X (the l dimension)
+constexpr int PRO_THREADS = 256;
+
+__device__ __forceinline__ float load_g(const void* g, int64_t idx, int is_bf16) {
+  return is_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(g)[idx])
+                 : reinterpret_cast<const float*>(g)[idx];
+}
+
+template <typename XT>
+__device__ __forceinline__ XT to_x(float v);
+template <>
+__device__ __forceinline__ float to_x<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 to_x<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// One CTA = one 32 x 128 tile of X (s x l view) of one matrix.
+// The value that enters the sum of squares is the fp32 U (before bf16 rounding).
+template <typename XT>
+__global__ void __launch_bounds__(PRO_THREADS)
+prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_mode, int g_is_bf16,
+                float beta, int nesterov, XT* __restrict__ X, int64_t ldx, float* __restrict__ partials,
+                int tiles_j, int n_part) {
+  __shared__ float tile[PRO_TJ][PRO_TI + 1];
+  __shared__ float red[PRO_THREADS / 32];
+  const int mat = blockIdx.y;
+  const MatDesc d = mats[mat];
+  const int ti = blockIdx.x / tiles_j, tj = blockIdx.x % tiles_j;
+  const int64_t i0 = (int64_t)ti * PRO_TI, j0 = (int64_t)tj * PRO_TJ;
+  XT* Xm = X + (int64_t)mat * s * ldx;
+  float ss = 0.f;
+  const int tid = threadIdx.x;
+
+  auto produce = [&](int64_t idx) -> float {   // idx: element index in the tensor's own layout
+    float u;
+    if (src_mode == SRC_MUON) {
+      const float g = load_g(d.g, idx, g_is_bf16);
+      const float mn = fmaf(beta, d.m[idx], g);
+      d.m[idx] = mn;
+      u = nesterov ? fmaf(beta, mn, g) : mn;
+    } else if (src_mode == SRC_RAW_F32) {
+      u = reinterpret_cast<const float*>(d.g)[idx];
+    } else {
+      u = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(d.g)[idx]);
+    }
+    return u;
+  };
+
+  if (!d.transposed) {
+    // tensor is s x l: X[i][j] = T[i][j]; lanes run along j
+    const int tx = tid & 31, ty = tid >> 5;   // 32 x 8
+#pragma unroll
+    for (int r = 0; r < PRO_TI / 8; ++r) {
+      const int64_t i = i0 + ty + r * 8;
+      if (i >= s) continue;
+#pragma unroll
+      for (int q = 0; q < PRO_TJ / 32; ++q) {
+        const int64_t j = j0 + tx + q * 32;
+        if (j < l) {
+          const float u = produce(i * l + j);
+          ss = fmaf(u, u, ss);
+          Xm[i * ldx + j] = to_x<XT>(u);
+        }
+      }
+    }
+  } else {
+    // tensor is l x s: X[i][j] = T[j][i]; read with lanes along i, write with lanes along j
+    const int tx = tid & 31, ty = tid >> 5;
+#pragma unroll 4
+    for (int r = 0; r < PRO_TJ / 8; ++r) {
+      const int jj = ty + r * 8;
+      const int64_t j = j0 + jj, i = i0 + tx;
+      float u = 0.f;
+      if (j < l && i < s) {
+        u = produce(j * s + i);
+        ss = fmaf(u, u, ss);
+      }
+      tile[jj][tx] = u;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < PRO_TI / 8; ++r) {
+      const int ii = ty + r * 8;
+      const int64_t i = i0 + ii;
+      if (i >= s) continue;
+#pragma unroll
+      for (int q = 0; q < PRO_TJ / 32; ++q) {
+        const int jj = tx + q * 32;
+        const int64_t j = j0 + jj;
+        if (j < l) Xm[i * ldx + j] = to_x<XT>(tile[jj][ii]);
+      }
+    }
+  }
+  // deterministic block reduction
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  if (tid == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < PRO_THREADS / 32; ++w) t += red[w];
+    partials[(int64_t)mat * n_part + blockIdx.x] = t;
+  }
+}
+
+__global__ void finalize_scales_kernel(const float* __restrict__ partials, int n_part, int n_mats,
+                                       float eps, float2* __restrict__ scales) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= n_mats) return;
+  const float* p = partials + (int64_t)warp * n_part;
+  double acc = 0.0;
+  for (int i = lane; i < n_part; i += 32) acc += (double)p[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const double r = 1.0 / (sqrt(acc) + (double)eps);
+    scales[warp] = make_float2((float)(r * r), (float)r);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// AdamW
+// ---------------------------------------------------------------------------
+constexpr int ADAM_THREADS = 256;
+
+__device__ __forceinline__ int find_adam_seg(const AdamSeg* __restrict__ segs, int n, int64_t unit) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (segs[mid].unit_begin <= unit) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ void adam_elem(float g, float& m, float& v, float& th, float beta1,
+                                          float beta2, float eps, const AdamSeg& s) {
+  m = fmaf(beta1, m, (1.0f - beta1) * g);
+  v = fmaf(beta2, v, (1.0f - beta2) * g * g);
+  const float mh = m * s.inv_bc1;
+  const float denom = fmaf(sqrtf(v), s.inv_sqrt_bc2, eps);
+  th = th - fmaf(s.lr, __fdiv_rn(mh, denom), s.lr_wd * th);
+}
+
+__global__ void __launch_bounds__(ADAM_THREADS)
+adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int g_is_bf16, float beta1,
+             float beta2, float eps) {
+  for (int64_t unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+    const int si = find_adam_seg(segs, n_segs, unit);
+    const AdamSeg s = segs[si];
+    const int64_t base = (unit - s.unit_begin) * ADAM_UNIT;
+    int64_t cnt = s.n - base;
+    if (cnt > ADAM_UNIT) cnt = ADAM_UNIT;
+    const bool vec = !g_is_bf16 &&
+                     ((((uintptr_t)s.g | (uintptr_t)s.m | (uintptr_t)s.v | (uintptr_t)s.theta) & 15) == 0);
+    if (vec) {
+      const float4* g4 = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(s.g) + base);
+      float4* m4 = reinterpret_cast<float4*>(s.m + base);
+      float4* v4 = reinterpret_cast<float4*>(s.v + base);
+      float4* t4 = reinterpret_cast<float4*>(s.theta + base);
+      const int n4 = (int)(cnt >> 2);
+#pragma unroll
+      for (int r = 0; r < ADAM_UNIT / 4 / ADAM_THREADS; ++r) {
+        const int i = threadIdx.x + r * ADAM_THREADS;
+        if (i < n4) {
+          const float4 g = __ldcs(g4 + i);
+          float4 m = m4[i], v = v4[i], t = t4[i];
+          adam_elem(g.x, m.x, v.x, t.x, beta1, beta2, eps, s);
+          adam_elem(g.y, m.y, v.y, t.y, beta1, beta2, eps, s);
+          adam_elem(g.z, m.z, v.z, t.z, beta1, beta2, eps, s);
+          adam_elem(g.w, m.w, v.w, t.w, beta1, beta2, eps, s);
+          m4[i] = m; v4[i] = v; t4[i] = t;
+        }
+      }
+      for (int64_t i = (int64_t)n4 * 4 + threadIdx.x; i < cnt; i += ADAM_THREADS) {
+        float g = reinterpret_cast<const float*>(s.g)[base + i];
+        float m = s.m[base + i], v = s.v[base + i], t = s.theta[base + i];
+        adam_elem(g, m, v, t, beta1, beta2, eps, s);
+        s.m[base + i] = m; s.v[base + i] = v; s.theta[base + i] = t;
+      }
+    } else {
+      for (int64_t i = threadIdx.x; i < cnt; i += ADAM_THREADS) {
+        float g = load_g(s.g, base + i, g_is_bf16);
+        float m = s.m[base + i], v = s.v[base + i], t = s.theta[base + i];
+        adam_elem(g, m, v, t, beta1, beta2, eps, s);
+        s.m[base + i] = m; s.v[base + i] = v; s.theta[base + i] = t;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+int prologue_partials_per_matrix(int64_t s, int64_t l) {
+  return (int)(((s + PRO_TI - 1) / PRO_TI) * ((l + PRO_TJ - 1) / PRO_TJ));
+}
+
+void launch_prologue(cudaStream_t st, const MatDesc* mats, int n_mats, int64_t s, int64_t l,
+                     int src_mode, int g_is_bf16, float beta, int nesterov, void* X, int x_is_f32,
+                     int64_t ldx, float* partials) {
+  if (n_mats <= 0) return;
+  const int tiles_j = (int)((l + PRO_TJ - 1) / PRO_TJ);
+  const int n_part = prologue_partials_per_matrix(s, l);
+  for (int m0 = 0; m0 < n_mats; m0 += 65535) {
+    const int nm = (n_mats - m0 < 65535) ? (n_mats - m0) : 65535;
+    dim3 grid((unsigned)n_part, (unsigned)nm);
+    if (x_is_f32)
+      prologue_kernel<float><<<grid, PRO_THREADS, 0, st>>>(
+          mats + m0, s, l, src_mode, g_is_bf16, beta, nesterov,
+          reinterpret_cast<float*>(X) + (int64_t)m0 * s * ldx, ldx, partials + (int64_t)m0 * n_part,
+          tiles_j, n_part);
+    else
+      prologue_kernel<__nv_bfloat16><<<grid, PRO_THREADS, 0, st>>>(
+          mats + m0, s, l, src_mode, g_is_bf16, beta, nesterov,
+          reinterpret_cast<__nv_bfloat16*>(X) + (int64_t)m0 * s * ldx, ldx,
+          partials + (int64_t)m0 * n_part, tiles_j, n_part);
+  }
+}
+
+void launch_finalize_scales(cudaStream_t st, const float* partials, int n_part, int n_mats, float eps,
+                            float2* scales) {
+  if (n_mats <= 0) return;
+  const int threads = 128;
+  const int blocks = (n_mats * 32 + threads - 1) / threads;
+  finalize_scales_kernel<<<blocks, threads, 0, st>>>(partials, n_part, n_mats, eps, scales);
+}
+
+void launch_adamw(cudaStream_t st, const AdamSeg* segs, int n_segs, int64_t n_units, int g_is_bf16,
+                  float beta1, float beta2, float eps) {
+  if (n_units <= 0 || n_segs <= 0) return;
+  int64_t blocks = n_units < (int64_t)148 * 16 ? n_units : (int64_t)148 * 16;
+  adamw_kernel<<<(unsigned)blocks, ADAM_THREADS, 0, st>>>(segs, n_segs, n_units, g_is_bf16, beta1,
+                                                          beta2, eps);
+}
+
+}  // namespace muloco

@@ -1,0 +1,102 @@
+// Internal declarations shared by the CUDA translation units of libmuloco.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/muloco.h"
+
+namespace muloco {
+
+// Device status word bits (OR-ed by kernels, read by muloco_sync_status).
+enum : int { ST_NONFINITE = 1, ST_TIMEOUT = 2, ST_BOUNDS = 4 };
+
+// ---------------------------------------------------------------------------
+// Muon path: one entry per (worker, hidden matrix) of a chunk.
+// The Newton-Schulz workspace always holds X as s x l with s <= l; a matrix
+// stored with rows > cols enters and leaves through its transpose.
+// ---------------------------------------------------------------------------
+struct MatDesc {
+  const void* g;   // gradient (fp32 or bf16), tensor layout rows x cols; or raw X for the standalone call
+  float* m;        // Muon momentum (fp32), tensor layout; NULL for the standalone call
+  void* w;         // parameters W (fp32, updated in place) or output O of the standalone call
+  float lr_eff;    // eta' = lr * lr_scale * lr_mult
+  float wd_term;   // eta_wd * lambda * wd_mult (multiplies W)
+  int32_t transposed;  // 1: tensor is l x s (rows > cols)
+  int32_t pad;
+};
+
+enum SrcMode : int { SRC_MUON = 0, SRC_RAW_F32 = 1, SRC_RAW_BF16 = 2 };
+enum SinkMode : int { SINK_UPDATE_W = 0, SINK_STORE_F32 = 1, SINK_STORE_BF16 = 2 };
+
+// prologue: m <- beta m + g; U -> workspace X (bf16 or fp32, s x ldx per slot); partial sums of U^2.
+// partial layout: partials[slot * n_part + tile], n_part = ceil(s/32) * ceil(l/128).
+void launch_prologue(cudaStream_t st, const MatDesc* mats, int n_mats, int64_t s, int64_t l,
+                     int src_mode, int g_is_bf16, float beta, int nesterov, void* X, int x_is_f32,
+                     int64_t ldx, float* partials);
+int prologue_partials_per_matrix(int64_t s, int64_t l);
+// scales[slot] = { r*r, r } with r = 1 / (sqrt(sum partials) + eps)
+void launch_finalize_scales(cudaStream_t st, const float* partials, int n_part, int n_mats,
+                            float eps, float2* scales);
+
+// fp32 Newton-Schulz engine (CUDA cores).  One call = one of the three products
+// of an iteration for all matrices of a chunk.
+enum GemmKind : int { GEMM_GRAM = 0, GEMM_POLY = 1, GEMM_APPLY = 2, GEMM_FINAL = 3 };
+struct NsIterArgs {
+  float a, b, c;            // quintic coefficients
+  const float2* scales;     // per-slot {r^2, r}; NULL: no scaling in this call
+  const MatDesc* mats;      // for GEMM_FINAL (sink)
+  int sink_mode;
+  int* status;
+};
+void launch_ns_fp32(cudaStream_t st, int kind, int n_mats, int64_t s, int64_t l, const float* X,
+                    int64_t ldx, const float* A, const float* B, int64_t lds, float* Aout,
+                    float* Bout, float* Xout, const NsIterArgs& args);
+
+// bf16 tensor-core engine (tcgen05 / TMEM / TMA); see ns_tc.cu.
+struct TcGroupPlan;   // opaque per-shape-group plan (tensor maps, tile lists)
+TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1, int64_t ldx,
+                            void* A, void* B, int64_t lds, char* err, size_t errlen);
+void tc_plan_destroy(TcGroupPlan*);
+// runs one product for the first n_mats slots; xin selects which X buffer is the input (0/1)
+cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* plan, int kind, int n_mats, int xin,
+                      const NsIterArgs& args);
+int tc_num_sms();
+
+// AdamW: one entry per (worker, tensor).
+struct AdamSeg {
+  const void* g;
+  float* m;
+  float* v;
+  float* theta;
+  int64_t n;
+  int64_t unit_begin;   // first work unit (of ADAM_UNIT elements) of this segment
+  float lr;             // alpha
+  float lr_wd;          // alpha * lambda * wd_mult
+  float inv_bc1;        // 1 / (1 - beta1^t) (1 if no bias correction)
+  float inv_sqrt_bc2;   // 1 / sqrt(1 - beta2^t)
+};
+constexpr int ADAM_UNIT = 2048;
+void launch_adamw(cudaStream_t st, const AdamSeg* segs, int n_segs, int64_t n_units, int g_is_bf16,
+                  float beta1, float beta2, float eps);
+
+// Outer sync: one entry per tensor of the fragment.
+struct SyncSeg {
+  float* theta_g;
+  float* u;
+  int64_t rows, cols;
+  int64_t nblk;         // blocks per row
+  int64_t unit_begin;   // first block-unit of this segment
+  int64_t rep_index;    // index of this tensor's first replica pointer in the replica table
+};
+void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
+                       int K, int64_t n_units, int block, int quant_bits, float outer_lr,
+                       float mu, int* status, int n_sms);
+void launch_pseudogradient(cudaStream_t st, const float* theta_g, float* const* replicas, int K,
+                           int64_t n, float* psi_out);
+void launch_quantize(cudaStream_t st, const float* psi, int64_t rows, int64_t cols, int block,
+                     int bits, int8_t* codes, float* scales, float* dequant, int* status);
+void launch_broadcast_init(cudaStream_t st, const float* src, float* const* dst_table, int K,
+                           int64_t n);
+
+}  // namespace muloco

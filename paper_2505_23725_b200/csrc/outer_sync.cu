@@ -1,0 +1,312 @@
+// Outer synchronisation (Algorithm 1 lines 9-13, Eqs. 2-3) as ONE pass over memory:
+// pseudogradient over the K replicas, optional per-block quantise->dequantise,
+// Nesterov outer step, broadcast into the K replicas.  Pure HBM streaming:
+// (K+2) fp32 reads and (K+2) fp32 writes per parameter.
+//
+// Work unit = one block of `block` (<= 128) consecutive elements of one row,
+// handled by one warp, four elements per lane (128-bit accesses when the row
+// pitch allows).  A CTA owns a contiguous span of units so that each of the
+// K+2 streams is read in long runs.
+#include <float.h>
+
+#include "internal.h"
+
+namespace muloco {
+
+namespace {
+
+constexpr int SYNC_THREADS = 256;
+constexpr int SYNC_WARPS = SYNC_THREADS / 32;
+
+__device__ __forceinline__ int find_seg(const SyncSeg* __restrict__ segs, int n, int64_t unit) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (segs[mid].unit_begin <= unit) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Quantise -> dequantise the (up to) four values of this lane; the block is the
+// whole warp.  Exact fp32 operations, no contraction: amax, inv = qmax / amax,
+// q = rint(x * inv) clamped, scale = amax / qmax, x^ = q * scale.
+template <int QB>
+__device__ __forceinline__ void quant_dequant4(float (&x)[4], int nvalid, int (&q)[4], float& scale,
+                                               bool& bad) {
+  constexpr float qmax = (QB == 8) ? 127.0f : 7.0f;
+  float lmax = 0.0f;
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if (e < nvalid) {
+      float a = fabsf(x[e]);
+      if (!(a <= FLT_MAX)) bad = true;
+      lmax = fmaxf(lmax, a);
+    }
+  const float amax = warp_max(lmax);
+  if (amax > 0.0f && amax <= FLT_MAX) {
+    const float inv = __fdiv_rn(qmax, amax);
+    scale = __fdiv_rn(amax, qmax);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float r = rintf(__fmul_rn(x[e], inv));
+      r = fminf(fmaxf(r, -qmax), qmax);
+      q[e] = (int)r;
+      x[e] = __fmul_rn(r, scale);
+    }
+  } else {
+    scale = 0.0f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { q[e] = 0; x[e] = 0.0f; }
+  }
+}
+
+__device__ __forceinline__ void load4(const float* __restrict__ p, bool vec, int nvalid, float (&v)[4]) {
+  if (vec) {
+    float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = (e < nvalid) ? __ldcs(p + e) : 0.0f;
+  }
+}
+
+__device__ __forceinline__ void store4(float* __restrict__ p, bool vec, int nvalid, const float (&v)[4]) {
+  if (vec) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(v[0], v[1], v[2], v[3]));
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (e < nvalid) __stcs(p + e, v[e]);
+  }
+}
+
+// KT > 0: K known at compile time (all replica loads in flight at once).
+template <int KT, int QB>
+__global__ void __launch_bounds__(SYNC_THREADS)
+outer_sync_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps,
+                  int Krt, int64_t n_units, int64_t units_per_cta, int block, float eta, float mu,
+                  float inv_k, int* __restrict__ status) {
+  const int K = (KT > 0) ? KT : Krt;
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t cta_begin = (int64_t)blockIdx.x * units_per_cta;
+  int64_t cta_end = cta_begin + units_per_cta;
+  if (cta_end > n_units) cta_end = n_units;
+  bool bad = false;
+
+  int64_t unit = cta_begin + warp;
+  if (unit < cta_end) {
+    int seg = find_seg(segs, n_segs, unit);
+    SyncSeg s = segs[seg];
+    int64_t seg_end = (seg + 1 < n_segs) ? segs[seg + 1].unit_begin : n_units;
+    bool aligned = ((s.cols & 3) == 0) && ((((uintptr_t)s.theta_g | (uintptr_t)s.u) & 15) == 0);
+    for (; unit < cta_end; unit += SYNC_WARPS) {
+      while (unit >= seg_end) {
+        ++seg;
+        s = segs[seg];
+        seg_end = (seg + 1 < n_segs) ? segs[seg + 1].unit_begin : n_units;
+        aligned = ((s.cols & 3) == 0) && ((((uintptr_t)s.theta_g | (uintptr_t)s.u) & 15) == 0);
+      }
+      const int64_t ul = unit - s.unit_begin;
+      const int64_t row = ul / s.nblk;
+      const int64_t blk = ul - row * s.nblk;
+      const int64_t col0 = blk * block + lane * 4;
+      int64_t blk_end = (blk + 1) * block;
+      if (blk_end > s.cols) blk_end = s.cols;
+      int nvalid = (int)(blk_end - col0);
+      nvalid = nvalid < 0 ? 0 : (nvalid > 4 ? 4 : nvalid);
+      const int64_t off = row * s.cols + col0;
+      float* const* rp = reps + s.rep_index;
+
+      float tg[4], uu[4], acc[4] = {0.f, 0.f, 0.f, 0.f};
+      bool vec = aligned && nvalid == 4;
+      if (nvalid > 0) {
+        if (KT > 0) {
+          float r[KT > 0 ? KT : 1][4];
+          bool v2 = vec;
+#pragma unroll
+          for (int k = 0; k < KT; ++k) v2 = v2 && ((((uintptr_t)rp[k]) & 15) == 0);
+          vec = v2;
+          load4(s.theta_g + off, vec, nvalid, tg);
+          load4(s.u + off, vec, nvalid, uu);
+#pragma unroll
+          for (int k = 0; k < KT; ++k) load4(rp[k] + off, vec, nvalid, r[k]);
+#pragma unroll
+          for (int k = 0; k < KT; ++k)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], __fsub_rn(tg[e], r[k][e]));
+        } else {
+          for (int k = 0; k < K; ++k) vec = vec && ((((uintptr_t)rp[k]) & 15) == 0);
+          load4(s.theta_g + off, vec, nvalid, tg);
+          load4(s.u + off, vec, nvalid, uu);
+          for (int k0 = 0; k0 < K; k0 += 4) {
+            float r[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (k0 + j < K) load4(rp[k0 + j] + off, vec, nvalid, r[j]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (k0 + j < K)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], __fsub_rn(tg[e], r[j][e]));
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { tg[e] = 0.f; uu[e] = 0.f; }
+      }
+      float psi[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) psi[e] = __fmul_rn(acc[e], inv_k);
+      if (QB != 0) {
+        int q[4]; float sc;
+        quant_dequant4<(QB == 0 ? 8 : QB)>(psi, nvalid, q, sc, bad);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (e < nvalid && !(fabsf(psi[e]) <= FLT_MAX)) bad = true;
+      }
+      if (nvalid > 0) {
+        float un[4], tn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float ep = eta * psi[e];
+          un[e] = fmaf(mu, uu[e], ep);
+          tn[e] = tg[e] - fmaf(mu, un[e], ep);
+        }
+        store4(s.u + off, vec, nvalid, un);
+        store4(s.theta_g + off, vec, nvalid, tn);
+        for (int k = 0; k < K; ++k) store4(rp[k] + off, vec, nvalid, tn);
+      }
+    }
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
+}
+
+__global__ void pseudograd_kernel(const float* __restrict__ tg, float* const* __restrict__ reps, int K,
+                                  int64_t n, float inv_k, float* __restrict__ out) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) {
+    const float t = tg[i];
+    float acc = 0.f;
+    for (int k = 0; k < K; ++k) acc = __fadd_rn(acc, __fsub_rn(t, reps[k][i]));
+    out[i] = __fmul_rn(acc, inv_k);
+  }
+}
+
+template <int QB>
+__global__ void quantize_kernel(const float* __restrict__ psi, int64_t rows, int64_t cols, int block,
+                                int64_t nblk, int8_t* __restrict__ codes, float* __restrict__ scales,
+                                float* __restrict__ deq, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n_units = rows * nblk;
+  bool bad = false;
+  for (int64_t unit = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < n_units;
+       unit += (int64_t)gridDim.x * (blockDim.x >> 5)) {
+    const int64_t row = unit / nblk, blk = unit - row * nblk;
+    const int64_t col0 = blk * block + lane * 4;
+    int64_t blk_end = (blk + 1) * block;
+    if (blk_end > cols) blk_end = cols;
+    int nvalid = (int)(blk_end - col0);
+    nvalid = nvalid < 0 ? 0 : (nvalid > 4 ? 4 : nvalid);
+    const int64_t off = row * cols + col0;
+    float x[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) x[e] = (e < nvalid) ? psi[off + e] : 0.f;
+    int q[4]; float sc;
+    quant_dequant4<QB>(x, nvalid, q, sc, bad);
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (e < nvalid) {
+        if (codes) codes[off + e] = (int8_t)q[e];
+        if (deq) deq[off + e] = x[e];
+      }
+    if (scales && lane == 0) scales[row * nblk + blk] = sc;
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
+}
+
+__global__ void broadcast_kernel(const float* __restrict__ src, float* const* __restrict__ dst, int K,
+                                 int64_t n) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) {
+    const float v = src[i];
+    for (int k = 0; k < K; ++k) dst[k][i] = v;
+  }
+}
+
+template <int QB>
+void launch_sync_q(cudaStream_t st, dim3 grid, const SyncSeg* segs, int n_segs, float* const* reps,
+                   int K, int64_t n_units, int64_t upc, int block, float eta, float mu, float inv_k,
+                   int* status) {
+#define MULOCO_SYNC_CASE(KT)                                                                      \
+  outer_sync_kernel<KT, QB><<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, reps, K, n_units, upc,   \
+                                                           block, eta, mu, inv_k, status)
+  switch (K) {
+    case 1: MULOCO_SYNC_CASE(1); break;
+    case 2: MULOCO_SYNC_CASE(2); break;
+    case 4: MULOCO_SYNC_CASE(4); break;
+    case 8: MULOCO_SYNC_CASE(8); break;
+    case 16: MULOCO_SYNC_CASE(16); break;
+    default: MULOCO_SYNC_CASE(0); break;
+  }
+#undef MULOCO_SYNC_CASE
+}
+
+}  // namespace
+
+void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
+                       int K, int64_t n_units, int block, int quant_bits, float outer_lr, float mu,
+                       int* status, int n_sms) {
+  if (n_units <= 0) return;
+  // persistent-style grid: a multiple of the SM count, each CTA a contiguous span
+  int64_t ctas = (int64_t)n_sms * 8;
+  int64_t min_units = SYNC_WARPS * 4;   // at least a few units per warp
+  if (ctas * min_units > n_units) ctas = (n_units + min_units - 1) / min_units;
+  if (ctas < 1) ctas = 1;
+  const int64_t upc = (n_units + ctas - 1) / ctas;
+  ctas = (n_units + upc - 1) / upc;
+  const float inv_k = 1.0f / (float)K;
+  dim3 grid((unsigned)ctas);
+  if (quant_bits == 8)
+    launch_sync_q<8>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+  else if (quant_bits == 4)
+    launch_sync_q<4>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+  else
+    launch_sync_q<0>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+}
+
+void launch_pseudogradient(cudaStream_t st, const float* theta_g, float* const* replicas, int K,
+                           int64_t n, float* psi_out) {
+  if (n <= 0) return;
+  int blocks = (int)((n + 255) / 256 < 2048 ? (n + 255) / 256 : 2048);
+  pseudograd_kernel<<<blocks, 256, 0, st>>>(theta_g, replicas, K, n, 1.0f / (float)K, psi_out);
+}
+
+void launch_quantize(cudaStream_t st, const float* psi, int64_t rows, int64_t cols, int block,
+                     int bits, int8_t* codes, float* scales, float* dequant, int* status) {
+  const int64_t nblk = (cols + block - 1) / block;
+  const int64_t n_units = rows * nblk;
+  if (n_units <= 0) return;
+  int blocks = (int)((n_units + 7) / 8 < 4096 ? (n_units + 7) / 8 : 4096);
+  if (bits == 8)
+    quantize_kernel<8><<<blocks, 256, 0, st>>>(psi, rows, cols, block, nblk, codes, scales, dequant, status);
+  else
+    quantize_kernel<4><<<blocks, 256, 0, st>>>(psi, rows, cols, block, nblk, codes, scales, dequant, status);
+}
+
+void launch_broadcast_init(cudaStream_t st, const float* src, float* const* dst_table, int K, int64_t n) {
+  if (n <= 0) return;
+  int blocks = (int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096);
+  broadcast_kernel<<<blocks, 256, 0, st>>>(src, dst_table, K, n);
+}
+
+}  // namespace muloco

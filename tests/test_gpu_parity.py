@@ -1,0 +1,372 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+the same seeded inputs.  Tolerances: quantised codes bit-exact; fp32
+elementwise steps 1e-6 relative; Newton-Schulz 1e-4 (fp32 mode) and 2e-2 (bf16
+mode) relative Frobenius."""
+import numpy as np
+import pytest
+
+from oracle import muloco_oracle as O
+from paper_2505_23725_b200 import configs, synth
+from helpers import assert_close_1e6, gpu_for, oracle_for, relfro, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+# ---------------------------------------------------------------------------
+# configuration 0 in full: every buffer after H = 2 inner steps and one sync
+# ---------------------------------------------------------------------------
+def test_cfg0_full_round_fp32_mode():
+    w = configs.workload(0)
+    rng = np.random.default_rng(w.seed)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init)
+    before = [[_np(gpu.theta_k[k][i]).copy() for i in range(gpu.n)] for k in range(w.K)]
+    for k in range(w.K):                      # create() broadcast theta_g into the replicas
+        for i in range(gpu.n):
+            assert np.array_equal(before[k][i], init[i])
+    for h in range(w.H):
+        gs = [synth.host_gradients(rng, w.tensors) for _ in range(w.K)]
+        gpu.inner_step(-1, to_dev(gs))
+        orc.inner_step_all(gs)
+    gpu.sync_status()
+    for k in range(w.K):
+        for i in range(gpu.n):
+            assert_close_1e6(_np(gpu.state1[k][i]), orc.state1[k][i], f"momentum k={k} i={i}")
+            d_gpu = _np(gpu.theta_k[k][i]).astype(np.float64) - init[i]
+            d_ref = orc.theta_k[k][i].astype(np.float64) - init[i]
+            assert relfro(d_gpu, d_ref) < 1e-4, f"inner delta k={k} i={i}: {relfro(d_gpu, d_ref):.3e}"
+    # outer sync from the GPU's own replicas vs the oracle fed the same replicas
+    for k in range(w.K):
+        for i in range(gpu.n):
+            orc.theta_k[k][i][...] = _np(gpu.theta_k[k][i])
+    gpu.outer_sync(-1)
+    orc.outer_sync(-1)
+    gpu.sync_status()
+    for i in range(gpu.n):
+        assert_close_1e6(_np(gpu.theta_g[i]), orc.theta_g[i], f"theta_g {i}")
+        assert_close_1e6(_np(gpu.outer_u[i]), orc.outer_u[i], f"u {i}")
+        for k in range(w.K):
+            assert np.array_equal(_np(gpu.theta_k[k][i]), _np(gpu.theta_g[i]))
+    gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# Newton-Schulz on its own
+# ---------------------------------------------------------------------------
+NS_SHAPES = [(1, 128, 128), (2, 128, 352), (2, 352, 128), (1, 256, 512), (3, 768, 768), (1, 200, 300),
+             (2, 100, 72), (1, 64, 64), (1, 8, 24), (2, 1024, 2816), (1, 2816, 1024), (5, 384, 640)]
+
+
+@pytest.fixture(scope="module")
+def ns_ctx():
+    w = configs.Workload("ns-only", K=1, H=1, J=1, tensors=[], muon_lr=0.02, muon_beta=0.95, muon_wd=0.0,
+                         outer_lr=1.0, outer_momentum=0.0)
+    g = gpu_for(w, [])
+    yield g
+    g.close()
+
+
+@pytest.mark.parametrize("batch,m,n", NS_SHAPES)
+@pytest.mark.parametrize("mode,tol", [("fp32", 1e-4), ("bf16", 2e-2)])
+def test_newton_schulz_vs_oracle(ns_ctx, batch, m, n, mode, tol):
+    import torch
+    rng = np.random.default_rng(1000 + m * 7 + n)
+    X = np.stack([synth.lowrank_plus_noise(rng, m, n) * (10.0 ** rng.uniform(-3, 3)) for _ in range(batch)])
+    out = _np(ns_ctx.newton_schulz(torch.from_numpy(X).cuda(), ns_mode=mode))
+    ns_ctx.sync_status()
+    for b in range(batch):
+        ref = O.newton_schulz(X[b])
+        assert relfro(out[b], ref) < tol, f"{mode} {m}x{n} batch {b}: {relfro(out[b], ref):.3e}"
+
+
+def test_newton_schulz_bf16_io_and_zero_matrix(ns_ctx):
+    import torch
+    rng = np.random.default_rng(5)
+    X = torch.from_numpy(synth.lowrank_plus_noise(rng, 256, 384)).cuda().to(torch.bfloat16)
+    out = ns_ctx.newton_schulz(X, out_dtype=torch.bfloat16, ns_mode="bf16")
+    ref = O.newton_schulz(_np(X.float()))
+    assert relfro(_np(out.float()), ref) < 2e-2
+    Z = torch.zeros(2, 128, 256, device="cuda")
+    for mode in ("fp32", "bf16"):
+        oz = _np(ns_ctx.newton_schulz(Z, ns_mode=mode))
+        assert np.all(oz == 0)
+    ns_ctx.sync_status()
+
+
+# ---------------------------------------------------------------------------
+# outer sync
+# ---------------------------------------------------------------------------
+def _sync_workload(K, quant, shapes, J=1):
+    ts = [configs.Tensor(f"t{i}", r, c, configs.MUON if min(r, c) > 1 else configs.ADAMW, i % J)
+          for i, (r, c) in enumerate(shapes)]
+    return configs.Workload("sync", K=K, H=J, J=J, tensors=ts, muon_lr=0.02, muon_beta=0.9, muon_wd=0.0,
+                            outer_lr=0.7, outer_momentum=0.9, quant_bits=quant, ns_mode="fp32")
+
+
+SYNC_SHAPES = [(128, 352), (352, 128), (5, 100), (3, 7), (1, 1000), (1, 129), (64, 128), (257, 131)]
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 8, 16])
+@pytest.mark.parametrize("quant", [0, 8, 4])
+def test_outer_sync_vs_oracle(K, quant):
+    import torch
+    w = _sync_workload(K, quant, SYNC_SHAPES)
+    rng = np.random.default_rng(77 + K + quant)
+    init = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) * 0.02 for t in w.tensors]
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init)
+    for rnd in range(2):                                   # two syncs: the momentum buffer is exercised
+        for k in range(K):
+            for i, t in enumerate(w.tensors):
+                drift = (rng.standard_normal((t.rows, t.cols)) * 10.0 ** rng.uniform(-4, -1)).astype(np.float32)
+                if i == 2 and rnd == 0:
+                    drift[1, :] = 0.0                      # a block whose pseudogradient is exactly zero
+                orc.theta_k[k][i][...] = orc.theta_g[i] + drift
+                gpu.theta_k[k][i].copy_(torch.from_numpy(orc.theta_k[k][i]).cuda())
+        # the pseudogradient itself: bitwise equal to the fp32 same-order definition
+        for i in range(gpu.n):
+            psi = _np(gpu.pseudogradient(i))
+            ref32 = O.pseudogradient_f32(orc.theta_g[i], [orc.theta_k[k][i] for k in range(K)])
+            assert np.array_equal(psi, ref32), f"psi tensor {i}"
+            if quant:
+                codes, scales, deq = gpu.quantize(torch.from_numpy(psi).cuda(), quant)
+                rc, rs, rd = O.quantize_blocks(ref32, quant, 128)
+                assert np.array_equal(_np(codes), rc), f"codes tensor {i}"
+                assert np.array_equal(_np(scales), rs) and np.array_equal(_np(deq), rd)
+        gpu.outer_sync(-1)
+        orc.outer_sync(-1)
+        gpu.sync_status()
+        for i in range(gpu.n):
+            assert_close_1e6(_np(gpu.theta_g[i]), orc.theta_g[i], f"theta_g {i} round {rnd}")
+            assert_close_1e6(_np(gpu.outer_u[i]), orc.outer_u[i], f"u {i} round {rnd}")
+            for k in range(K):
+                assert np.array_equal(_np(gpu.theta_k[k][i]), _np(gpu.theta_g[i]))
+            # keep the two sides in lock-step for the next round
+            orc.theta_g[i][...] = _np(gpu.theta_g[i]); orc.outer_u[i][...] = _np(gpu.outer_u[i])
+    gpu.close()
+
+
+def test_streaming_fragments_touch_only_their_tensors():
+    import torch
+    J = 4
+    w = _sync_workload(4, 8, [(64, 128)] * 8, J=J)
+    w.H = 8
+    rng = np.random.default_rng(3)
+    init = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) for t in w.tensors]
+    gpu = gpu_for(w, init)
+    for k in range(4):
+        for i in range(gpu.n):
+            gpu.theta_k[k][i].add_(0.01 * (k + 1))
+    due = {t: gpu.fragments_due(t) for t in range(0, 17)}
+    assert due[0] == [] and due[2] == [0] and due[4] == [1] and due[6] == [2] and due[8] == [3] and due[10] == [0]
+    assert [t for t in range(1, 9) if due[t]] == [2, 4, 6, 8]
+    for f in range(J):
+        snap_g = [_np(v).copy() for v in gpu.theta_g]
+        snap_k = [_np(v).copy() for v in gpu.theta_k[0]]
+        gpu.outer_sync(f)
+        gpu.sync_status()
+        for i, t in enumerate(w.tensors):
+            changed = not np.array_equal(_np(gpu.theta_g[i]), snap_g[i])
+            assert changed == (t.fragment == f)
+            if t.fragment != f:
+                assert np.array_equal(_np(gpu.theta_k[0][i]), snap_k[i])
+    gpu.close()
+
+
+def test_nonfinite_pseudogradient_is_reported():
+    from paper_2505_23725_b200 import binding
+    w = _sync_workload(2, 8, [(4, 128)])
+    gpu = gpu_for(w, [np.zeros((4, 128), np.float32)])
+    gpu.theta_k[1][0][2, 5] = float("inf")
+    gpu.outer_sync(-1)
+    with pytest.raises(binding.MulocoError) as e:
+        gpu.sync_status()
+    assert e.value.status == binding.ENONFINITE
+    gpu.sync_status()          # the status word was cleared
+    gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# AdamW and the full inner step on a mixed model
+# ---------------------------------------------------------------------------
+def test_adamw_and_mixed_inner_steps():
+    w = configs.mini_workload(K=3, H=3, L=1, d=64, F=96, vocab=500, norms=True, ns_mode="fp32",
+                              adam_lr=3e-3, adam_wd=0.05)
+    rng = np.random.default_rng(12)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init)
+    for h in range(3):
+        gs = [synth.host_gradients(rng, w.tensors) for _ in range(w.K)]
+        if h == 1:      # single-worker calls in a scrambled order must equal the batched call
+            dev = to_dev(gs)
+            for k in (2, 0, 1):
+                gpu.inner_step(k, dev[k], lr_scale=0.5)
+                orc.inner_step(k, gs[k], lr_scale=0.5)
+        else:
+            gpu.inner_step(-1, to_dev(gs))
+            orc.inner_step_all(gs)
+        gpu.sync_status()
+        for k in range(w.K):
+            for i, t in enumerate(w.tensors):
+                if t.kind == configs.ADAMW:
+                    assert_close_1e6(_np(gpu.state1[k][i]), orc.state1[k][i], f"adam m h={h}")
+                    assert_close_1e6(_np(gpu.state2[k][i]), orc.state2[k][i], f"adam v h={h}")
+                    assert_close_1e6(_np(gpu.theta_k[k][i]), orc.theta_k[k][i], f"adam theta h={h} {t.name}")
+                else:
+                    assert relfro(_np(gpu.theta_k[k][i]), orc.theta_k[k][i]) < 1e-5
+                # lock-step
+                orc.theta_k[k][i][...] = _np(gpu.theta_k[k][i])
+                orc.state1[k][i][...] = _np(gpu.state1[k][i])
+                if t.kind == configs.ADAMW:
+                    orc.state2[k][i][...] = _np(gpu.state2[k][i])
+    gpu.close()
+
+
+def test_batched_equals_per_worker_calls_bitwise():
+    w = configs.mini_workload(K=4, H=2, L=1, d=128, F=352, vocab=300, norms=True, ns_mode="bf16")
+    rng = np.random.default_rng(13)
+    init = synth.init_weights(rng, w.tensors)
+    a = gpu_for(w, init); b = gpu_for(w, init)
+    for h in range(2):
+        dev = to_dev([synth.host_gradients(rng, w.tensors) for _ in range(w.K)])
+        a.inner_step(-1, dev)
+        for k in (3, 1, 0, 2):
+            b.inner_step(k, dev[k])
+    a.sync_status(); b.sync_status()
+    for k in range(w.K):
+        for i in range(a.n):
+            assert np.array_equal(_np(a.theta_k[k][i]), _np(b.theta_k[k][i]))
+            assert np.array_equal(_np(a.state1[k][i]), _np(b.state1[k][i]))
+    a.close(); b.close()
+
+
+def test_bf16_mode_inner_step_vs_oracle():
+    w = configs.mini_workload(K=2, H=2, L=1, d=256, F=640, ns_mode="bf16")
+    rng = np.random.default_rng(14)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init)
+    for h in range(2):
+        gs = [synth.host_gradients(rng, w.tensors) for _ in range(w.K)]
+        prev = [[_np(gpu.theta_k[k][i]).copy() for i in range(gpu.n)] for k in range(w.K)]
+        gpu.inner_step(-1, to_dev(gs))
+        orc.inner_step_all(gs)
+        gpu.sync_status()
+        for k in range(w.K):
+            for i in range(gpu.n):
+                assert_close_1e6(_np(gpu.state1[k][i]), orc.state1[k][i], "momentum")
+                d_gpu = _np(gpu.theta_k[k][i]).astype(np.float64) - prev[k][i]
+                d_ref = orc.theta_k[k][i].astype(np.float64) - prev[k][i]
+                assert relfro(d_gpu, d_ref) < 2e-2, f"h={h} k={k} i={i}: {relfro(d_gpu, d_ref):.3e}"
+                orc.theta_k[k][i][...] = _np(gpu.theta_k[k][i])
+                orc.state1[k][i][...] = _np(gpu.state1[k][i])
+    gpu.close()
+
+
+def test_k1_outer_identity_on_gpu():
+    w = configs.mini_workload(K=1, H=2, L=1, d=64, F=96, ns_mode="fp32", outer_lr=1.0, outer_momentum=0.0)
+    rng = np.random.default_rng(15)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    for h in range(2):
+        gpu.inner_step(-1, to_dev([synth.host_gradients(rng, w.tensors)]))
+    plain = [_np(v).copy() for v in gpu.theta_k[0]]
+    gpu.outer_sync(-1)
+    gpu.sync_status()
+    for i in range(gpu.n):
+        got = _np(gpu.theta_g[i])
+        # theta_g - fl(theta_g - theta_1): exact when the two are within a factor of two,
+        # otherwise off by at most one rounding at the magnitude of the larger of the two
+        tol = np.spacing(np.maximum(np.abs(init[i]), np.abs(plain[i])))
+        assert np.all(np.abs(got.astype(np.float64) - plain[i]) <= tol)
+        assert np.mean(got == plain[i]) > 0.9
+        assert np.array_equal(_np(gpu.theta_k[0][i]), got)
+    gpu.close()
+
+
+def test_identical_gradients_pseudogradient_equals_single_delta():
+    w = configs.mini_workload(K=4, H=1, L=1, d=64, F=96, ns_mode="fp32")
+    rng = np.random.default_rng(16)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    g = synth.host_gradients(rng, w.tensors)
+    gpu.inner_step(-1, to_dev([g] * 4))
+    gpu.sync_status()
+    for i in range(gpu.n):
+        for k in range(1, 4):
+            assert np.array_equal(_np(gpu.theta_k[k][i]), _np(gpu.theta_k[0][i]))
+        delta = init[i] - _np(gpu.theta_k[0][i])
+        assert np.array_equal(_np(gpu.pseudogradient(i)), delta)
+    gpu.close()
+
+
+def test_state_blob_roundtrip_and_resume():
+    w = configs.mini_workload(K=2, H=2, L=1, d=64, F=96, vocab=200, norms=True, ns_mode="fp32")
+    rng = np.random.default_rng(17)
+    init = synth.init_weights(rng, w.tensors)
+    gs = [to_dev([synth.host_gradients(rng, w.tensors) for _ in range(2)]) for _ in range(4)]
+    a = gpu_for(w, init)
+    for h in range(4):
+        a.inner_step(-1, gs[h])
+    b = gpu_for(w, init)
+    for h in range(2):
+        b.inner_step(-1, gs[h])
+    blob = b.get_state()
+    c = gpu_for(w, init)
+    for k in range(2):
+        for i in range(c.n):
+            c.theta_k[k][i].copy_(b.theta_k[k][i]); c.state1[k][i].copy_(b.state1[k][i])
+            if c.state2[k][i] is not None:
+                c.state2[k][i].copy_(b.state2[k][i])
+    c.set_state(blob)
+    for h in range(2, 4):
+        c.inner_step(-1, gs[h])
+    a.sync_status(); c.sync_status()
+    for k in range(2):
+        for i in range(a.n):
+            assert np.array_equal(_np(a.theta_k[k][i]), _np(c.theta_k[k][i]))
+    from paper_2505_23725_b200 import binding
+    with pytest.raises(binding.MulocoError):
+        c.set_state(blob[:-8])
+    a.close(); b.close(); c.close()
+
+
+def test_host_entry_points_match_device_entry_points():
+    import torch
+    w = configs.mini_workload(K=2, H=1, L=1, d=64, F=96, vocab=100, norms=True, ns_mode="fp32")
+    rng = np.random.default_rng(18)
+    init = synth.init_weights(rng, w.tensors)
+    a = gpu_for(w, init); b = gpu_for(w, init)
+    gs = [synth.host_gradients(rng, w.tensors) for _ in range(2)]
+    a.inner_step(-1, to_dev(gs))
+    host = [[torch.from_numpy(g).pin_memory() for g in gk] for gk in gs]
+    b.inner_step_host(-1, host)
+    a.outer_sync(-1)
+    out = [torch.empty(t.rows, t.cols).pin_memory() for t in w.tensors]
+    b.outer_sync_host(-1, out)
+    a.sync_status(); b.sync_status()
+    for i in range(a.n):
+        assert np.array_equal(_np(a.theta_g[i]), _np(b.theta_g[i]))
+        assert np.array_equal(out[i].numpy(), _np(b.theta_g[i]))
+    a.close(); b.close()
+
+
+def test_argument_errors_are_reported_on_the_host():
+    from paper_2505_23725_b200 import binding
+    w = configs.mini_workload(K=2, H=4, J=3, L=1, d=64, F=96)
+    with pytest.raises(binding.MulocoError) as e:
+        gpu_for(w, None)
+    assert e.value.status == binding.EINVAL
+    w = configs.mini_workload(K=2, H=2, L=1, d=64, F=96)
+    gpu = gpu_for(w, None)
+    with pytest.raises(binding.MulocoError):
+        gpu.outer_sync(5)
+    with pytest.raises(binding.MulocoError):
+        gpu.inner_step(7, [gpu.theta_g[i] for i in range(gpu.n)])
+    gpu.close()
