@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the MuLoCo optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--impl reference]
+
+One "step" is one full MuLoCo round of the workload: H inner steps of all K
+workers (Muon prologue + Newton-Schulz + update, AdamW) followed by the outer
+synchronisation of every fragment at its scheduled step -- every row of the hot
+path runs in each timed step.  metric = optimizer-step parameter updates per
+second, K * N_params * H per round.  Prints ONE JSON line on rank 0.
+
+Default workload: benchmark configuration 2 (416M-shaped, K=16, H=30), the one
+the target is quoted on.  With --gpus N > 1 every rank runs its own independent
+K-worker problem on its own GPU (weak scaling, no data-path collective: the
+method keeps its K workers on one GPU).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "optimizer-step params/sec (inner Muon + outer sync) at K workers"
+UNIT = "param-updates/s"
+
+# DRAM traffic (bytes) per credited FLOP of the Newton-Schulz GEMM kernels, from the
+# ncu capture summarised in profiles/; None until a capture exists.
+NS_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "200"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx = float(f[2])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        med = sm[len(sm) // 2] if sm else None
+        return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_cores():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle_sample(w, seed=0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload:
+    one layer's hidden matrices for one worker (Muon), a 2^20-element AdamW slice,
+    and the outer sync of one hidden matrix shape set over all K replicas.  Returns
+    the extrapolated parameter updates per second over a full round and a
+    description of the sample."""
+    import numpy as np
+    from oracle import muloco_oracle as O
+    from paper_2505_23725_b200 import configs
+
+    rng = np.random.default_rng(seed)
+    layer = [t for t in w.tensors if t.kind == configs.MUON and t.name.startswith("l0.")]
+    pm = sum(t.numel for t in layer)
+    Ws = [(0.02 * rng.standard_normal((t.rows, t.cols))).astype(np.float32) for t in layer]
+    Ms = [np.zeros_like(x) for x in Ws]
+    Gs = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) for t in layer]
+    t0 = time.perf_counter()
+    for W, M, G in zip(Ws, Ms, Gs):
+        O.muon_step(W, M, G, lr=w.muon_lr, beta=w.muon_beta, wd=w.muon_wd, nesterov=w.muon_nesterov)
+    t_muon = time.perf_counter() - t0
+    pa = 1 << 20
+    th = rng.standard_normal(pa).astype(np.float32); m = np.zeros_like(th); v = np.zeros_like(th)
+    g = rng.standard_normal(pa).astype(np.float32)
+    t0 = time.perf_counter()
+    O.adamw_step(th, m, v, g, t=1, lr=w.muon_lr, wd=w.muon_wd)
+    t_adam = time.perf_counter() - t0
+    t_sync, ps = 0.0, 0
+    for t in layer[:2] + layer[-1:]:
+        tg = (0.02 * rng.standard_normal((t.rows, t.cols))).astype(np.float32)
+        u = np.zeros_like(tg)
+        reps = [tg + (1e-3 * rng.standard_normal(tg.shape)).astype(np.float32) for _ in range(w.K)]
+        t0 = time.perf_counter()
+        if w.quant_bits:
+            _, _, psi = O.quantize_blocks(O.pseudogradient_f32(tg, reps), w.quant_bits, w.quant_block)
+        else:
+            psi = O.pseudogradient(tg, reps)
+        O.outer_nesterov(tg, u, psi, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum)
+        for r in reps:
+            r[...] = tg
+        t_sync += time.perf_counter() - t0
+        ps += t.numel
+    n_muon = w.n_muon_params
+    n_adam = w.n_params - n_muon
+    t_round = w.H * w.K * (n_muon / pm * t_muon + n_adam / pa * t_adam) + w.n_params / ps * t_sync
+    value = w.K * w.n_params * w.H / t_round
+    sample = (f"one layer x one worker Muon step ({len(layer)} matrices, {pm} params, {t_muon:.2f} s), "
+              f"AdamW on 2^20 elements ({t_adam:.3f} s), outer sync of {ps} params x K={w.K} replicas "
+              f"({t_sync:.2f} s); extrapolated linearly to a full round of H={w.H} steps")
+    return value, sample, t_muon + t_adam + t_sync
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle on the host cores, same metric and config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals, tot = [], 0.0
+    sample = ""
+    for _ in range(args.warmup):
+        time_oracle_sample(w)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        v, sample, _ = time_oracle_sample(w)
+        vals.append(v)
+    tot = time.perf_counter() - t0
+    value = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_cores(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(w, args):
+    return {"workload": f"configs[{args.config}] {w.name}: K={w.K} H={w.H} J={w.J}, {w.n_params} params/replica "
+                        f"({w.n_muon_params} on Muon), quant={w.quant_bits or 'none'}, NS {w.ns_mode}",
+            "step": "one round = H inner steps (all K workers) + scheduled outer syncs",
+            "l2": "inputs_larger_than_l2", "parallelism": "K replicas on one GPU; ranks independent"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workspace-gb", type=float, default=0.0)
+    args = ap.parse_args()
+
+    from paper_2505_23725_b200 import configs
+    w = configs.workload(args.config)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2505_23725_b200 import binding, synth
+    import __graft_entry__ as entry
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if rank == 0:
+        entry.build()
+    distributed = world > 1
+    if distributed:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+        dist.barrier()
+    dev = f"cuda:{local_rank}"
+    torch.cuda.set_device(dev)
+
+    opt = binding.MuLoCo(w, dev, init_seed=w.seed + 1000 * rank, alloc_grads=True,
+                         workspace_bytes=int(args.workspace_gb * (1 << 30)))
+    synth.torch_fill_gradients(opt.grads, w.tensors, w.K, w.seed + 17 * rank, opt.device)
+    torch.cuda.synchronize()
+
+    def one_round(t0):
+        """H inner steps with the streaming schedule; returns the step counter."""
+        t = t0
+        for _ in range(w.H):
+            opt.inner_step(-1, None, 1.0)
+            t += 1
+            for f in opt.fragments_due(t):
+                opt.outer_sync(f)
+        return t
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    t = 0
+    for _ in range(args.warmup):
+        t = one_round(t)
+    opt.sync_status()
+    opt.set_timing(True)
+    opt.get_timings()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(opt.stream)
+    for _ in range(args.steps):
+        t = one_round(t)
+    e1.record(opt.stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    phases, launches = opt.get_timings()
+    opt.set_timing(False)
+    opt.sync_status()
+    if distributed:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_per_step = ms_total / args.steps
+    units_per_round = w.K * w.n_params * w.H
+    value = world * units_per_round / (ms_per_step * 1e-3)
+
+    # ---- roofline of the dominant kernel (Newton-Schulz tensor-core GEMMs) ----------------
+    peaks = load_peaks()
+    inner_steps = args.steps * w.H
+    ns_ms_per_inner = phases["ns"] / inner_steps
+    ns_tflops = w.ns_flops_credited() / (ns_ms_per_inner * 1e-3) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    ns_launches_per_inner = None
+    roofline = {"bound": "tensor", "kernel": "ns_tc_kernel (Gram / polynomial / apply GEMMs of Newton-Schulz)",
+                "achieved": ns_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": ns_tflops / peak_tf,
+                "peak_source": f"{peaks['source']} sustained bf16 matmul", "traffic": NS_TRAFFIC_BYTES_PER_LAUNCH,
+                "flops_convention": "credited 5*(4 s^2 l + 2 s^3) per matrix; symmetric products run upper-triangle tiles only",
+                "ms_per_inner_step": ns_ms_per_inner}
+    n_sync_rounds = args.steps
+    sync_gbs = w.sync_bytes() * n_sync_rounds / (phases["sync"] * 1e-3) / 1e9 if phases["sync"] > 0 else None
+    n_adam = w.n_params - w.n_muon_params
+    adam_bytes = n_adam * w.K * (28.0 if w.grad_dtype == "f32" else 26.0) * inner_steps
+    adam_gbs = adam_bytes / (phases["adamw"] * 1e-3) / 1e9 if phases["adamw"] > 0 else None
+    pro_bytes = w.n_muon_params * w.K * (14.0 if w.grad_dtype == "f32" else 12.0) * inner_steps
+    pro_gbs = pro_bytes / (phases["prologue"] * 1e-3) / 1e9 if phases["prologue"] > 0 else None
+    phase_report = {
+        "ms_per_round": {k: v / args.steps for k, v in phases.items()},
+        "ns_tflops_credited": ns_tflops, "ns_frac_of_burst_peak": ns_tflops / peaks["bf16_tflops"],
+        "sync_gbs": sync_gbs, "sync_frac_of_hbm": (sync_gbs / peaks["hbm_gbs"]) if sync_gbs else None,
+        "adamw_gbs": adam_gbs, "adamw_frac_of_hbm": (adam_gbs / peaks["hbm_gbs"]) if adam_gbs else None,
+        "prologue_gbs": pro_gbs, "hbm_peak_gbs": peaks["hbm_gbs"],
+    }
+
+    # ---- end to end through the host-buffer entry points ----------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(opt, w, torch, dist if distributed else None, world)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, sample, _ = time_oracle_sample(w)
+        cpu = {"value": v, "unit": UNIT, "cores": oracle_cores(), "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if w.ns_mode == "bf16" else "f32", "data": "synthetic",
+                "config": workload_config(w, args), "clocks": clocks, "e2e": e2e,
+                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "phases": phase_report}
+        print(json.dumps(line))
+    opt.close()
+    if distributed:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(opt, w, torch, dist, world):
+    """The same round through muloco_inner_step_host / muloco_outer_sync_host: every inner
+    step copies that step's gradients from pinned host memory, every sync reads the new
+    global parameters back to the host.  One warm-up inner step, one timed round."""
+    import psutil
+    elt = 2 if w.grad_dtype == "bf16" else 4
+    set_bytes = opt.flat_numel * elt
+    avail = psutil.virtual_memory().available
+    n_sets = w.K if set_bytes * w.K * 1.5 < avail else 1
+    # drop the device-resident gradients: in this mode they come from the host each step
+    opt.grads = None; opt.flat_grads = None; opt._grad_table_all = None
+    torch.cuda.empty_cache()
+    host_flat = [torch.empty(opt.flat_numel, dtype=opt.gdtype).pin_memory() for _ in range(n_sets)]
+    for hf in host_flat:
+        hf.normal_(0.0, 0.01)
+    host = [[host_flat[k % n_sets][o:o + t.numel].view(t.rows, t.cols) for o, t in zip(opt.offsets, w.tensors)]
+            for k in range(w.K)]
+    out_flat = torch.empty(opt.flat_numel, dtype=torch.float32).pin_memory()
+    out = [out_flat[o:o + t.numel].view(t.rows, t.cols) for o, t in zip(opt.offsets, w.tensors)]
+    opt.inner_step_host(-1, host, 1.0)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(opt.stream)
+    t = 0
+    d2h = 0
+    for _ in range(w.H):
+        opt.inner_step_host(-1, host, 1.0)
+        t += 1
+        for f in opt.fragments_due(t):
+            opt.outer_sync_host(f, out)
+            d2h += sum(tt.numel for tt in w.tensors if tt.fragment == f) * 4
+    e1.record(opt.stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist:
+        tt = torch.tensor([ms], device=opt.device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    opt.sync_status()
+    h2d = w.n_params * elt * w.K * w.H
+    return {"value": world * w.K * w.n_params * w.H / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "rounds_timed": 1, "host_grad_sets": n_sets}
+
+
+if __name__ == "__main__":
+    main()

@@ -149,7 +149,7 @@ class MuLoCo:
 
     def __init__(self, workload: _cfg.Workload, device="cuda:0", init: Optional[Sequence[np.ndarray]] = None,
                  workspace_bytes: int = 0, ns_mode: Optional[str] = None, stream=None, alloc_grads: bool = False,
-                 **config_overrides):
+                 init_seed: Optional[int] = None, **config_overrides):
         import torch
 
         self.torch = torch
@@ -183,9 +183,18 @@ class MuLoCo:
         if init is not None:
             for i, a in enumerate(init):
                 self.theta_g[i].copy_(torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev))
+        elif init_seed is not None:
+            # device-side initial weights for the large configurations: N(0, 0.02^2), gains = 1
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(init_seed)
+            self.flat_theta_g.normal_(0.0, 0.02, generator=gen)
+            for i, t in enumerate(workload.tensors):
+                if t.init == "ones":
+                    self.theta_g[i].fill_(1.0)
         self.gdtype = torch.bfloat16 if workload.grad_dtype == "bf16" else torch.float32
         self.flat_grads = None
         self.grads = None
+        self._grad_table_all = None
         if alloc_grads:
             self.alloc_grads()
 
@@ -215,7 +224,6 @@ class MuLoCo:
             msg = self.lib.muloco_last_error(None).decode()
             self.ctx = None
             raise MulocoError(st, msg)
-        self._grad_table_all = None
 
     # -- helpers --------------------------------------------------------------
     def _views(self, flat):
