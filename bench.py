@@ -201,7 +201,12 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workspace-gb", type=float, default=0.0)
+    ap.add_argument("--ns-only", type=int, nargs=3, metavar=("BATCH", "ROWS", "COLS"), default=None,
+                    help="kernel study: time muloco_newton_schulz (bf16 engine) on a batch of one shape")
     args = ap.parse_args()
+    if args.ns_only:
+        run_ns_only(args)
+        return
 
     from paper_2505_23725_b200 import configs
     w = configs.workload(args.config)
@@ -325,6 +330,39 @@ def main():
     if distributed:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_ns_only(args):
+    """Small case for kernel studies and ncu captures: the standalone Newton-Schulz call
+    (15 tensor-core launches per call) on BATCH matrices of ROWS x COLS."""
+    import torch
+    from paper_2505_23725_b200 import binding, configs
+    import __graft_entry__ as entry
+    entry.build()
+    batch, rows, cols = args.ns_only
+    w = configs.Workload("ns-only", K=1, H=1, J=1, tensors=[], muon_lr=0.02, muon_beta=0.95, muon_wd=0.0,
+                         outer_lr=1.0, outer_momentum=0.0)
+    opt = binding.MuLoCo(w, "cuda:0", init=[], workspace_bytes=int(args.workspace_gb * (1 << 30)))
+    gen = torch.Generator(device="cuda"); gen.manual_seed(0)
+    X = torch.randn(batch, rows, cols, device="cuda", generator=gen).to(torch.bfloat16)
+    for _ in range(args.warmup):
+        opt.newton_schulz(X, out_dtype=torch.bfloat16)
+    opt.set_timing(True); opt.get_timings()
+    torch.cuda.synchronize()
+    for _ in range(args.steps):
+        opt.newton_schulz(X, out_dtype=torch.bfloat16)
+    ph, launches = opt.get_timings()
+    opt.sync_status()
+    s, l = min(rows, cols), max(rows, cols)
+    flops = batch * 5.0 * (4.0 * s * s * l + 2.0 * s ** 3)
+    ms = ph["ns"] / args.steps
+    peaks = load_peaks()
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({"ns_only": [batch, rows, cols], "ms_per_call": ms, "tflops_credited": tf,
+                      "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+                      "frac_of_burst_peak": tf / peaks["bf16_tflops"], "prologue_ms": ph["prologue"] / args.steps,
+                      "launches": int(launches)}))
+    opt.close()
 
 
 def run_e2e(opt, w, torch, dist, world):

@@ -167,6 +167,40 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* ctx, const void* X, in
                                    int32_t o_dtype, int32_t batch, int64_t rows, int64_t cols,
                                    int32_t ns_mode);
 
+/* Size of the fixed scratch behind muloco_newton_schulz_static (bytes). */
+#define MULOCO_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* Newton-Schulz for callers that must not allocate device memory.  (The paper has
+ * no counterpart: this is a packaging variant of muloco_newton_schulz in its fp32
+ * mode, with the paper's coefficients, 5 steps and eps = 1e-7.)
+ *
+ * Who needs it: code running where a device allocation is off limits -- after a
+ * framework's caching allocator has taken the whole GPU, so that a raw cudaMalloc
+ * may fail or fragment the pool, or inside a latency-critical loop that cannot pay
+ * for the device-wide synchronisation that allocating and freeing imply.  This call
+ * needs no context (creating one allocates) and calls no cudaMalloc, cudaFree or
+ * other allocating routine: its scratch is a fixed array of
+ * MULOCO_STATIC_SCRATCH_BYTES inside the library image, which every GPU that loads
+ * the library holds until the process exits.
+ *
+ * X: [batch][rows][cols] float32 device input, O: same shape float32 device output
+ * (must not overlap X); batch <= 64.  The scratch must hold, per matrix with
+ * s = min(rows, cols), l = max(rows, cols): 2*s*l + 2*s*s floats (each row padded
+ * to 8 elements) plus small tables; a request that does not fit returns
+ * MULOCO_ESHAPE and explains the sizes in errbuf -- use muloco_newton_schulz then.
+ * errbuf (host, may be NULL) receives a NUL-terminated message on failure.
+ * The work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default stream) of
+ * the CURRENT device.
+ *
+ * The first call on each device resolves the scratch's device address (once per
+ * device, that device being current); make that first call before starting any
+ * stream capture.  All calls on a device share the one scratch array, which keeps
+ * whatever the last call left in it: calls whose GPU work overlaps in time
+ * (different streams or threads) race with each other -- serialise them. */
+MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, float* O, int32_t batch,
+                                                     int64_t rows, int64_t cols, void* cuda_stream,
+                                                     char* errbuf, size_t errbuf_len);
+
 /* The block quantiser on its own (the benchmark's per-block absmax form of the
  * linear quantisation of Section 2, "Compressed Communication"): psi is a
  * rows x cols float32 matrix; writes, where non-NULL, one int8 code per element

@@ -32,6 +32,7 @@ EXPORTS = [
     "muloco_outer_sync", "muloco_outer_sync_host", "muloco_fragments_due", "muloco_newton_schulz",
     "muloco_quantize", "muloco_pseudogradient", "muloco_get_state", "muloco_set_state",
     "muloco_set_timing", "muloco_get_timings", "muloco_sync_status", "muloco_last_error",
+    "muloco_newton_schulz_static",
 ]
 
 
@@ -97,12 +98,34 @@ def load_library():
     lib.muloco_sync_status.argtypes = [vp]
     lib.muloco_last_error.argtypes = [vp]
     lib.muloco_last_error.restype = C.c_char_p
+    lib.muloco_newton_schulz_static.argtypes = [vp, vp, i32, i64, i64, vp, C.c_char_p, C.c_size_t]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("muloco_destroy", "muloco_last_error"):
             fn.restype = i32
     _lib = lib
     return lib
+
+
+def newton_schulz_static(X, stream=None):
+    """muloco_newton_schulz_static: fp32 Newton-Schulz of a small [batch, rows, cols]
+    (or [rows, cols]) float32 CUDA tensor without any device allocation by the library
+    (the output tensor is allocated here, by torch, before the call).  For callers that
+    may not allocate; sizes beyond the library's fixed scratch raise MulocoError(ESHAPE)."""
+    import torch
+    lib = load_library()
+    x = (X if X.dim() == 3 else X.unsqueeze(0)).contiguous()
+    if x.dtype != torch.float32 or not x.is_cuda:
+        raise ValueError("expects a float32 CUDA tensor")
+    o = torch.empty_like(x)
+    st = stream if stream is not None else torch.cuda.current_stream(x.device)
+    err = C.create_string_buffer(256)
+    with torch.cuda.device(x.device):
+        rc = lib.muloco_newton_schulz_static(x.data_ptr(), o.data_ptr(), x.shape[0], x.shape[1], x.shape[2],
+                                             C.c_void_p(st.cuda_stream), err, 256)
+    if rc != OK:
+        raise MulocoError(rc, err.value.decode())
+    return o if X.dim() == 3 else o[0]
 
 
 def make_config(w: _cfg.Workload, workspace_bytes: int = 0, ns_mode: Optional[str] = None, **over) -> Config:
