@@ -6,19 +6,31 @@
 // (Section 2, "Muon": X_j = p(X X^T) X, p(x) = a x + b x^3 + c x^5) for every
 // matrix of a chunk; tiles of all matrices form one linear work list:
 //   GRAM  : A  = r^2 X X^T      symmetric: only tiles touching the upper triangle,
-//   POLY  : B  = b A + c A A    each stored directly and mirrored
+//   POLY  : B  = b A + c A A    each 128-block stored directly and mirrored
 //   APPLY : X' = r (a X + B X)
 //   FINAL : as APPLY, result goes to the parameter update / output sink
 // Operand forms: GRAM/POLY multiply a row-major matrix by its own transpose
 // (both operands K-major); APPLY needs X with the contraction index as the slow
 // axis, i.e. an MN-major B operand, so no transposed copy of X is ever made.
 //
+// Two tile shapes share one kernel body (template parameter CG):
+//   CG = 2 : a pair of CTAs on neighbouring SMs (a cluster of two) computes a
+//            256 x 256 tile with tcgen05.mma.cta_group::2.  Each CTA stages its
+//            own 128 rows of the left operand and HALF of the right operand, so
+//            a stage is 32 KB per SM for 256 x 256 x 64 of work.  The CTA of
+//            rank 0 issues the MMAs; every CTA drains its own 128 accumulator
+//            rows.  No load is multicast: each CTA fetches its own slabs.
+//   CG = 1 : one CTA, 128 x 128 tiles (matrices with at most 128 rows).
+//
 // CTA = 6 warps: warp 0 issues TMA loads, warp 1 allocates tensor memory and
-// issues the MMAs, warps 2-5 run the epilogue (one 32-lane quarter of the
-// accumulator each).  Two accumulators alternate so the epilogue of one tile
-// overlaps the main loop of the next.  Every wait is bounded: when one runs out
-// the kernel raises ST_TIMEOUT, all roles leave their loops, and the CTA frees
-// its tensor memory and returns.
+// (rank 0) issues the MMAs, warps 2-5 run the epilogue (one 32-lane quarter of
+// the accumulator each).  Two accumulators alternate so the epilogue of one
+// tile overlaps the main loop of the next.  The epilogue goes through shared
+// memory: the addend (A for POLY, X for APPLY) arrives by TMA, results leave as
+// bulk tensor stores of whole 32 x 64 blocks (and, for the symmetric products,
+// of the transposed block), so global memory only sees full lines.
+// Every wait is bounded: when one runs out the kernel raises ST_TIMEOUT, all
+// roles leave their loops, and the CTA frees its tensor memory and returns.
 #include <cuda.h>
 #include <stdio.h>
 #include <string.h>
@@ -32,31 +44,25 @@ namespace muloco {
 
 namespace {
 
-constexpr int BM = 128;          // tile rows (UMMA M)
+constexpr int BM = 128;          // rows per CTA (one CTA's share of UMMA M)
 constexpr int BK = 64;           // k slab per stage (64 bf16 = one 128-byte swizzle row)
 constexpr int UMMA_K = 16;
 constexpr int TC_THREADS = 192;
-constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
+constexpr int STAGES = 4;
+constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;        // 16 KB: 128 rows x 64 k
+constexpr uint32_t B_STAGE_BYTES = 128 * BK * 2;       // 16 KB: this CTA's 128 columns of the right operand
+constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr uint32_t EPI_BLOCK_BYTES = 32 * 64 * 2;      // one 32 x 64 bf16 block
+constexpr uint32_t EPI_WARP_BYTES = 6 * EPI_BLOCK_BYTES;   // addend x2, direct x2, mirrored x2
+constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_WARP_BYTES + 1024;   // + alignment slack
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
-
-template <int BN> struct TcCfg {
-  static constexpr int STAGES = (BN == 256) ? 4 : 6;
-  static constexpr uint32_t B_STAGE_BYTES = BN * BK * 2;
-  static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + alignment slack
-  static constexpr uint32_t TMEM_COLS = 2 * BN;                          // two accumulators
-};
 
 struct TcParams {
   int kind;
   int n_mats;
   int M, N, Kd;
   int n_tiles_per_mat;
-  const int2* tiles;
-  const __nv_bfloat16* Cin;
-  int64_t ldc, strideC;
-  __nv_bfloat16* D;
-  int64_t ldd, strideD;
+  const int2* tiles;          // (tile row, tile col) in units of 128*CG
   float a, b, c;
   const float2* scales;
   const MatDesc* mats;
@@ -69,21 +75,37 @@ struct TcParams {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n"
+               "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// arrive on a barrier given by its shared::cluster address (own CTA or the peer)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
@@ -111,6 +133,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// TMA load whose completion is counted on a barrier of this CTA.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1, int c2) {
   asm volatile(
@@ -118,20 +141,70 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// TMA load into this CTA's shared memory whose completion is counted on a barrier that may
+// live in the peer CTA of the pair (shared::cluster address).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+
+template <int CG>
+__device__ __forceinline__ void tc_commit(uint32_t bar_cluster_addr) {
+  if (CG == 1)
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+  else
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
+template <int CG>
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (CG == 1)
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem_addr, uint32_t cols) {
+  if (CG == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem_addr), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  } else {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem_addr), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+}
+template <int CG>
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t cols) {
+  if (CG == 1)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+  else
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
@@ -168,52 +241,75 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
 
 // ------------------------------- the kernel --------------------------------
-template <int BN, bool B_MN>
+// tmA/tmB : operand loads (left: K-major 64 x 128 boxes; right: K-major 64 x 128 or, for B_MN,
+//           MN-major 64 x 64 boxes)
+// tmC     : addend loads, 64 x 32 boxes (POLY: A, APPLY/FINAL: X)
+// tmD     : result stores, 64 x 32 boxes, 128-byte swizzle
+// tmT     : transposed result stores, 32 x 64 boxes, no swizzle (symmetric products)
+template <int CG, bool B_MN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-             const TcParams p) {
-  using Cfg = TcCfg<BN>;
-  constexpr int STAGES = Cfg::STAGES;
+             const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
+             const __grid_constant__ CUtensorMap tmT, const TcParams p) {
+  constexpr int BN = 128 * CG;                 // accumulator columns = tile columns
+  constexpr int TM = 128 * CG;                 // tile rows (over the CTA pair)
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+  constexpr int NCH = BN / 64;                 // 64-column epilogue blocks per tile
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_full[STAGES];
+  __shared__ __align__(8) uint64_t bar_full[STAGES];    // used in the CTA of rank 0
   __shared__ __align__(8) uint64_t bar_empty[STAGES];
   __shared__ __align__(8) uint64_t bar_tfull[2];
-  __shared__ __align__(8) uint64_t bar_tempty[2];
+  __shared__ __align__(8) uint64_t bar_tempty[2];       // used in the CTA of rank 0
+  __shared__ __align__(8) uint64_t bar_cin[4][2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile int abort_flag;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;
+  const int unit = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // tile worker index
+  const int n_units = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int total_tiles = p.n_mats * p.n_tiles_per_mat;
   const int num_kb = (p.Kd + BK - 1) / BK;
+  const bool sym = (p.kind == GEMM_GRAM || p.kind == GEMM_POLY);
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmT) : "memory");
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&bar_tfull[a]), 1);
-      mbar_init(smem_u32(&bar_tempty[a]), 4);
+      mbar_init(smem_u32(&bar_tempty[a]), 4 * CG);
     }
+    for (int w = 0; w < 4; ++w)
+      for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bar_cin[w][b]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(&tmem_base_slot)),
-                 "r"(Cfg::TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
+  if (warp == 1) tmem_alloc<CG>(smem_u32(&tmem_base_slot), TMEM_COLS);
   tc_fence_before();
-  __syncthreads();
+  if (CG == 2) cluster_sync_all(); else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -221,25 +317,45 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // ------------------------------ TMA producer ------------------------------
     uint32_t stage = 0, phase = 0;
     bool alive = true;
-    for (int tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x) {
+    for (int tile = unit; tile < total_tiles && alive; tile += n_units) {
       const int mat = tile / p.n_tiles_per_mat;
       const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
+      const bool same = sym && (tt.x == tt.y);     // diagonal tile: right slab == left slab
+      const int a_row = BM * (CG * tt.x + (int)rank);
+      const int b_off = TM * tt.y + 128 * (int)rank;
+      const uint32_t cta_bytes = A_STAGE_BYTES + (same ? 0u : B_STAGE_BYTES);
       for (int kb = 0; kb < num_kb && alive; ++kb) {
         if (lane == 0) {
           if (mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, &abort_flag)) {
-            const uint32_t full = smem_u32(&bar_full[stage]);
-            const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+            const uint32_t full_local = smem_u32(&bar_full[stage]);
+            const uint32_t sa = smem_base + stage * STAGE_BYTES;
             const uint32_t sb = sa + A_STAGE_BYTES;
-            mbar_expect_tx(full, Cfg::STAGE_BYTES);
-            tma_load_3d(sa, &tmA, full, kb * BK, tt.x * BM, mat);
-            if (!B_MN) {
+            if (CG == 1) {
+              mbar_expect_tx(full_local, cta_bytes);
+              tma_load_3d(sa, &tmA, full_local, kb * BK, a_row, mat);
+              if (!same) {
+                if (!B_MN) {
+                  tma_load_3d(sb, &tmB, full_local, kb * BK, b_off, mat);
+                } else {
 #pragma unroll
-              for (int h = 0; h < BN / 128; ++h)
-                tma_load_3d(sb + h * (128 * BK * 2), &tmB, full, kb * BK, tt.y * BN + h * 128, mat);
+                  for (int q = 0; q < 2; ++q)
+                    tma_load_3d(sb + q * (BK * 128), &tmB, full_local, b_off + q * 64, kb * BK, mat);
+                }
+              }
             } else {
+              // both CTAs' copies are counted on the barrier of rank 0, which expects the sum
+              const uint32_t full0 = map_to_rank(full_local, 0);
+              if (rank == 0) mbar_expect_tx(full_local, 2u * cta_bytes);
+              tma_load_3d_pair(sa, &tmA, full0, kb * BK, a_row, mat);
+              if (!same) {
+                if (!B_MN) {
+                  tma_load_3d_pair(sb, &tmB, full0, kb * BK, b_off, mat);
+                } else {
 #pragma unroll
-              for (int q = 0; q < BN / 64; ++q)
-                tma_load_3d(sb + q * (BK * 128), &tmB, full, tt.y * BN + q * 64, kb * BK, mat);
+                  for (int q = 0; q < 2; ++q)
+                    tma_load_3d_pair(sb + q * (BK * 128), &tmB, full0, b_off + q * 64, kb * BK, mat);
+                }
+              }
             }
           }
         }
@@ -250,173 +366,231 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
-    constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((B_MN ? 1u : 0u) << 16) |
-                               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-    uint32_t stage = 0, phase = 0;
-    int local_tile = 0;
-    bool alive = true;
-    for (int tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x, ++local_tile) {
-      const int acc = local_tile & 1;
-      const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
-      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-      if (lane == 0) {
-        if (mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, &abort_flag)) tc_fence_after();
-      }
-      __syncwarp();
-      alive = (abort_flag == 0);
-      for (int kb = 0; kb < num_kb && alive; ++kb) {
+    if (rank == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((B_MN ? 1u : 0u) << 16) |
+                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+      uint32_t stage = 0, phase = 0;
+      int local_tile = 0;
+      bool alive = true;
+      for (int tile = unit; tile < total_tiles && alive; tile += n_units, ++local_tile) {
+        const int mat = tile / p.n_tiles_per_mat;
+        const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
+        const bool same = sym && (tt.x == tt.y);
+        const int acc = local_tile & 1;
+        const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         if (lane == 0) {
-          if (mbar_wait(smem_u32(&bar_full[stage]), phase, &abort_flag)) {
-            tc_fence_after();
-            const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
-            const uint32_t sb = sa + A_STAGE_BYTES;
-#pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k) {
-              const uint64_t adesc = make_sdesc(sa + k * (UMMA_K * 2), 16, 1024);
-              const uint64_t bdesc = B_MN ? make_sdesc(sb + k * (UMMA_K * 128), BK * 128, 1024)
-                                          : make_sdesc(sb + k * (UMMA_K * 2), 16, 1024);
-              tc_mma_bf16(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-            }
-            tc_commit(smem_u32(&bar_empty[stage]));
-          }
+          if (mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, &abort_flag)) tc_fence_after();
         }
         __syncwarp();
         alive = (abort_flag == 0);
-        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        for (int kb = 0; kb < num_kb && alive; ++kb) {
+          if (lane == 0) {
+            if (mbar_wait(smem_u32(&bar_full[stage]), phase, &abort_flag)) {
+              tc_fence_after();
+              const uint32_t sa = smem_base + stage * STAGE_BYTES;
+              const uint32_t sb = same ? sa : sa + A_STAGE_BYTES;
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) {
+                const uint64_t adesc = make_sdesc(sa + k * (UMMA_K * 2), 16, 1024);
+                const uint64_t bdesc = B_MN ? make_sdesc(sb + k * (UMMA_K * 128), BK * 128, 1024)
+                                            : make_sdesc(sb + k * (UMMA_K * 2), 16, 1024);
+                tc_mma_bf16<CG>(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              }
+              const uint32_t e_local = smem_u32(&bar_empty[stage]);
+              tc_commit<CG>(e_local);
+              if (CG == 2) tc_commit<CG>(map_to_rank(e_local, 1));
+            }
+          }
+          __syncwarp();
+          alive = (abort_flag == 0);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (alive && lane == 0) {
+          const uint32_t t_local = smem_u32(&bar_tfull[acc]);
+          tc_commit<CG>(t_local);
+          if (CG == 2) tc_commit<CG>(map_to_rank(t_local, 1));
+        }
+        __syncwarp();
       }
-      if (alive && lane == 0) tc_commit(smem_u32(&bar_tfull[acc]));
-      __syncwarp();
     }
   } else {
     // -------------------------------- epilogue --------------------------------
     const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter+32)
-    const int row = quarter * 32 + lane;
+    const int ew = warp - 2;               // staging slot of this warp
+    const uint32_t epi = smem_base + STAGES * STAGE_BYTES + (uint32_t)ew * EPI_WARP_BYTES;
+    // staging blocks of this warp: addend 0/1, direct 0/1, mirrored 0/1
+    auto cin_buf = [&](uint32_t b) { return epi + b * EPI_BLOCK_BYTES; };
+    auto out_buf = [&](uint32_t b) { return epi + (2u + b) * EPI_BLOCK_BYTES; };
+    auto mir_buf = [&](uint32_t b) { return epi + (4u + b) * EPI_BLOCK_BYTES; };
+    const uint32_t cin_bar0 = smem_u32(&bar_cin[ew][0]);
+    auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
+    const bool has_cin = (p.kind != GEMM_GRAM);
+    const bool stores = (p.kind != GEMM_FINAL);
+    uint32_t cin_issued = 0, cin_used = 0, st_count = 0;
     int local_tile = 0;
     bool alive = true;
-    const bool sym = (p.kind == GEMM_GRAM || p.kind == GEMM_POLY);
-    for (int tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x, ++local_tile) {
+    for (int tile = unit; tile < total_tiles && alive; tile += n_units, ++local_tile) {
       const int acc = local_tile & 1;
       const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
       const int mat = tile / p.n_tiles_per_mat;
       const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
-      if (!mbar_wait(smem_u32(&bar_tfull[acc]), acc_phase, &abort_flag)) { alive = false; }
+      const int rb = CG * tt.x + (int)rank;                 // 128-row block of this CTA
+      const int gi0 = rb * BM + quarter * 32;               // first row of this warp
+      const int gi = gi0 + lane;
+      const bool row_ok = gi < p.M;
+      // 64-column blocks of this tile that this warp has to produce
+      uint32_t todo = 0;
+      if (gi0 < p.M) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const int gj0 = TM * tt.y + c * 64;
+          if (gj0 < p.N && !(sym && (gj0 >> 7) < rb)) todo |= 1u << c;   // lower-triangle blocks come from their mirror image
+        }
+      }
+      auto issue_cin = [&](int c) {
+        if (lane == 0) {
+          const uint32_t b = cin_issued & 1u;
+          mbar_expect_tx(cin_bar(b), EPI_BLOCK_BYTES);
+          tma_load_3d(cin_buf(b), &tmC, cin_bar(b), TM * tt.y + c * 64, gi0, mat);
+        }
+        ++cin_issued;
+      };
+      if (has_cin && todo) issue_cin(__ffs(todo) - 1);
+      if (!mbar_wait(smem_u32(&bar_tfull[acc]), acc_phase, &abort_flag)) alive = false;
       alive = __all_sync(0xffffffffu, alive);
       if (!alive) break;
       tc_fence_after();
-      const int64_t gi = (int64_t)tt.x * BM + row;
-      const bool row_ok = gi < p.M;
       float sc = 1.f;
       if (p.scales) sc = (p.kind == GEMM_GRAM) ? p.scales[mat].x : p.scales[mat].y;
-      const __nv_bfloat16* Cm = p.Cin ? p.Cin + (int64_t)mat * p.strideC : nullptr;
-      __nv_bfloat16* Dm = p.D ? p.D + (int64_t)mat * p.strideD : nullptr;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int64_t gj0 = (int64_t)tt.y * BN + c * 32;
-        if (gj0 >= p.N) break;                       // warp-uniform
-        const int cb = (int)(gj0 / BM);              // 128-column block of this chunk
-        if (sym && cb < tt.x) continue;              // lower-triangle block: its mirror image writes it
-        uint32_t v[32];
-        tc_ld32(t_row + (uint32_t)(c * 32), v);
-        float f[32];
+      while (todo) {
+        const int c = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int gj0 = TM * tt.y + c * 64;
+        const bool mirror = sym && ((gj0 >> 7) > rb);
+        if (has_cin) {
+          if (todo) issue_cin(__ffs(todo) - 1);
+          bool ok = mbar_wait(cin_bar(cin_used & 1u), (cin_used >> 1) & 1u, &abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) { alive = false; break; }
+        }
+        const uint32_t cbuf = cin_buf(cin_used & 1u);
+        const uint32_t obuf = out_buf(st_count & 1u);
+        const uint32_t mbuf = mir_buf(st_count & 1u);
+        if (stores) {
+          if (lane == 0) bulk_wait_read_1();     // the block stored two steps ago has left this buffer
+          __syncwarp();
+        }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]);
-        const bool full_chunk = (gj0 + 32 <= p.N);
-        // ---- addend -----------------------------------------------------------
-        if (p.kind != GEMM_GRAM) {
-          float add[32];
-          const bool vec_in = full_chunk && ((p.ldc & 7) == 0) && ((((uintptr_t)Cm) & 15) == 0);
-          if (row_ok) {
-            const __nv_bfloat16* src = Cm + gi * p.ldc + gj0;
-            if (vec_in) {
+        for (int h = 0; h < 2; ++h) {
+          uint32_t v[32];
+          tc_ld32(t_row + (uint32_t)(c * 64 + h * 32), v);
+          float f[32];
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const uint4 u = *reinterpret_cast<const uint4*>(src + q * 8);
-                add[q * 8 + 0] = bf16_lo(u.x); add[q * 8 + 1] = bf16_hi(u.x);
-                add[q * 8 + 2] = bf16_lo(u.y); add[q * 8 + 3] = bf16_hi(u.y);
-                add[q * 8 + 4] = bf16_lo(u.z); add[q * 8 + 5] = bf16_hi(u.z);
-                add[q * 8 + 6] = bf16_lo(u.w); add[q * 8 + 7] = bf16_hi(u.w);
-              }
+          for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]);
+          if (has_cin) {
+            float add[32];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 u = lds128(cbuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q) ^ (lane & 7)) << 4));
+              add[q * 8 + 0] = bf16_lo(u.x); add[q * 8 + 1] = bf16_hi(u.x);
+              add[q * 8 + 2] = bf16_lo(u.y); add[q * 8 + 3] = bf16_hi(u.y);
+              add[q * 8 + 4] = bf16_lo(u.z); add[q * 8 + 5] = bf16_hi(u.z);
+              add[q * 8 + 6] = bf16_lo(u.w); add[q * 8 + 7] = bf16_hi(u.w);
+            }
+            if (p.kind == GEMM_POLY) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) f[e] = fmaf(p.c, f[e], p.b * add[e]);
             } else {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) add[e] = (gj0 + e < p.N) ? __bfloat162float(src[e]) : 0.f;
+              for (int e = 0; e < 32; ++e) f[e] = sc * fmaf(p.a, add[e], f[e]);
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) add[e] = 0.f;
+            for (int e = 0; e < 32; ++e) f[e] *= sc;
           }
-          if (p.kind == GEMM_POLY) {
+          if (!stores) {
+            // ---- parameter update / output sink (fp32 tensor in its own layout) ----
+            const int gjh = gj0 + h * 32;
+            if (row_ok && gjh < p.N) {
+              const MatDesc d = p.mats[mat];
+              const bool full_chunk = (gjh + 32 <= p.N);
+              const bool fast = !d.transposed && p.sink_mode != SINK_STORE_BF16 && full_chunk &&
+                                ((p.l & 3) == 0) && ((((uintptr_t)d.w) & 15) == 0);
+              if (fast) {
+                float4* w4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(d.w) + (int64_t)gi * p.l + gjh);
+                if (p.sink_mode == SINK_UPDATE_W) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) f[e] = fmaf(p.c, f[e], p.b * add[e]);
-          } else {
+                  for (int q = 0; q < 8; ++q) {
+                    float4 w = w4[q];
+                    w.x = fmaf(-d.lr_eff, f[q * 4 + 0], fmaf(-d.wd_term, w.x, w.x));
+                    w.y = fmaf(-d.lr_eff, f[q * 4 + 1], fmaf(-d.wd_term, w.y, w.y));
+                    w.z = fmaf(-d.lr_eff, f[q * 4 + 2], fmaf(-d.wd_term, w.z, w.z));
+                    w.w = fmaf(-d.lr_eff, f[q * 4 + 3], fmaf(-d.wd_term, w.w, w.w));
+                    w4[q] = w;
+                  }
+                } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) f[e] = sc * fmaf(p.a, add[e], f[e]);
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) f[e] *= sc;
-        }
-        // ---- store --------------------------------------------------------------
-        if (p.kind == GEMM_FINAL) {
-          if (row_ok) {
-            const MatDesc d = p.mats[mat];
-            const bool fast = !d.transposed && p.sink_mode != SINK_STORE_BF16 && full_chunk &&
-                              ((p.l & 3) == 0) && ((((uintptr_t)d.w) & 15) == 0);
-            if (fast) {
-              float4* w4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(d.w) + gi * p.l + gj0);
-              if (p.sink_mode == SINK_UPDATE_W) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  float4 w = w4[q];
-                  w.x = fmaf(-d.lr_eff, f[q * 4 + 0], fmaf(-d.wd_term, w.x, w.x));
-                  w.y = fmaf(-d.lr_eff, f[q * 4 + 1], fmaf(-d.wd_term, w.y, w.y));
-                  w.z = fmaf(-d.lr_eff, f[q * 4 + 2], fmaf(-d.wd_term, w.z, w.z));
-                  w.w = fmaf(-d.lr_eff, f[q * 4 + 3], fmaf(-d.wd_term, w.w, w.w));
-                  w4[q] = w;
+                  for (int q = 0; q < 8; ++q)
+                    w4[q] = make_float4(f[q * 4 + 0], f[q * 4 + 1], f[q * 4 + 2], f[q * 4 + 3]);
                 }
               } else {
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
-                  w4[q] = make_float4(f[q * 4 + 0], f[q * 4 + 1], f[q * 4 + 2], f[q * 4 + 3]);
+                for (int e = 0; e < 32; ++e)
+                  if (gjh + e < p.N) sink_element(d, p.sink_mode, p.s, p.l, gi, gjh + e, f[e]);
               }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (gj0 + e < p.N) sink_element(d, p.sink_mode, p.s, p.l, gi, gj0 + e, f[e]);
             }
-          }
-        } else {
-          if (row_ok) {
-            __nv_bfloat16* dst = Dm + gi * p.ldd + gj0;
-            const bool vec_out = full_chunk && ((p.ldd & 7) == 0) && ((((uintptr_t)Dm) & 15) == 0);
-            if (vec_out) {
+          } else {
+            // ---- stage the bf16 block (and its transpose) for the bulk stores ----
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                uint4 u;
-                u.x = pack_bf16x2(f[q * 8 + 0], f[q * 8 + 1]);
-                u.y = pack_bf16x2(f[q * 8 + 2], f[q * 8 + 3]);
-                u.z = pack_bf16x2(f[q * 8 + 4], f[q * 8 + 5]);
-                u.w = pack_bf16x2(f[q * 8 + 6], f[q * 8 + 7]);
-                *reinterpret_cast<uint4*>(dst + q * 8) = u;
+            for (int q = 0; q < 4; ++q) {
+              uint4 u;
+              u.x = pack_bf16x2(f[q * 8 + 0], f[q * 8 + 1]);
+              u.y = pack_bf16x2(f[q * 8 + 2], f[q * 8 + 3]);
+              u.z = pack_bf16x2(f[q * 8 + 4], f[q * 8 + 5]);
+              u.w = pack_bf16x2(f[q * 8 + 6], f[q * 8 + 7]);
+              sts128(obuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q) ^ (lane & 7)) << 4), u);
+            }
+            if (mirror) {
+              // transposed block T[e][lane]: neighbouring lanes exchange one value so that
+              // each lane writes a packed pair of one transposed row
+              const bool odd = lane & 1;
+#pragma unroll
+              for (int e = 0; e < 32; e += 2) {
+                const float send = odd ? f[e] : f[e + 1];
+                const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                const uint32_t pk = odd ? pack_bf16x2(recv, f[e + 1]) : pack_bf16x2(f[e], recv);
+                const int trow = h * 32 + e + (odd ? 1 : 0);
+                sts32(mbuf + (uint32_t)trow * 64u + (uint32_t)((lane & ~1) * 2), pk);
               }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (gj0 + e < p.N) dst[e] = __float2bfloat16_rn(f[e]);
-            }
-            if (sym && cb > tt.x) {
-              // mirror image: D[j][i] = D[i][j]; lanes hold consecutive i
-#pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (gj0 + e < p.N) Dm[(gj0 + e) * p.ldd + gi] = __float2bfloat16_rn(f[e]);
             }
           }
         }
+        if (has_cin) ++cin_used;
+        if (stores) {
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(&tmD, obuf, gj0, gi0, mat);
+            if (mirror) tma_store_3d(&tmT, mbuf, gi0, gj0, mat);
+            bulk_commit();
+          }
+          ++st_count;
+        } else {
+          __syncwarp();
+        }
       }
+      if (!alive) break;
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[acc]));
+      if (lane == 0) {
+        const uint32_t te = smem_u32(&bar_tempty[acc]);
+        mbar_arrive_cluster(CG == 2 ? map_to_rank(te, 0) : te);
+      }
     }
+    if (lane == 0) bulk_wait_all();
   }
 
   // ------------------------------- teardown ----------------------------------
@@ -427,11 +601,10 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     if (threadIdx.x == 0) atomicOr(p.status, ST_TIMEOUT);
   }
   tc_fence_before();
-  __syncthreads();
+  if (CG == 2) cluster_sync_all(); else __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::TMEM_COLS)
-                 : "memory");
+    tmem_dealloc<CG>(tmem_base, TMEM_COLS);
   }
 }
 
@@ -455,7 +628,7 @@ EncodeTiledFn get_encode_fn() {
 
 // 3-D map over [n_slots][rows][cols] bf16 with row pitch ld; box = box_cols x box_rows x 1.
 bool encode_map(CUtensorMap* out, void* base, int64_t cols, int64_t rows, int64_t n_slots, int64_t ld,
-                int box_cols, int box_rows) {
+                int box_cols, int box_rows, bool swizzle128) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)n_slots};
@@ -463,25 +636,63 @@ bool encode_map(CUtensorMap* out, void* base, int64_t cols, int64_t rows, int64_
   cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
-template <int BN, bool B_MN>
-cudaError_t launch_one(cudaStream_t st, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p,
-                       int n_sms) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(ns_tc_kernel<BN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)TcCfg<BN>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    configured = true;
+struct Maps5 {
+  const CUtensorMap *a, *b, *c, *d, *t;
+};
+
+// Number of tile workers (CTAs for CG = 1, CTA pairs for CG = 2) that can be resident at once.
+template <int CG, bool B_MN>
+int resident_units(int n_sms, cudaError_t* err) {
+  static int cached = 0;
+  *err = cudaSuccess;
+  if (cached) return cached;
+  cudaError_t e = cudaFuncSetAttribute(ns_tc_kernel<CG, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES);
+  if (e != cudaSuccess) { *err = e; return 0; }
+  if (CG == 1) {
+    cached = n_sms;
+    return cached;
   }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)(n_sms / 2 * 2));
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = 0;
+  e = cudaOccupancyMaxActiveClusters(&n, ns_tc_kernel<CG, B_MN>, &cfg);
+  if (e != cudaSuccess) { *err = e; return 0; }
+  if (n < 1) { *err = cudaErrorLaunchOutOfResources; return 0; }
+  cached = n;
+  return cached;
+}
+
+template <int CG, bool B_MN>
+cudaError_t launch_one(cudaStream_t st, const Maps5& m, const TcParams& p, int n_sms) {
+  cudaError_t e;
+  const int units = resident_units<CG, B_MN>(n_sms, &e);
+  if (e != cudaSuccess) return e;
   const int total = p.n_mats * p.n_tiles_per_mat;
-  const int grid = total < n_sms ? total : n_sms;
-  ns_tc_kernel<BN, B_MN><<<grid, TC_THREADS, TcCfg<BN>::SMEM_BYTES, st>>>(a, b, p);
-  return cudaGetLastError();
+  const int workers = total < units ? total : units;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)(workers * CG));
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, ns_tc_kernel<CG, B_MN>, *m.a, *m.b, *m.c, *m.d, *m.t, p);
 }
 
 }  // namespace
@@ -489,11 +700,13 @@ cudaError_t launch_one(cudaStream_t st, const CUtensorMap& a, const CUtensorMap&
 struct TcGroupPlan {
   int64_t s, l, ldx, lds;
   int chunk;
+  int cg;                       // CTAs per tile worker (1 or 2)
   void* X[2];
   void* A;
   void* B;
-  CUtensorMap x_k[2], x_mn[2], a_k, b_k;
-  int bn_sym, bn_apply;
+  // loads: K-major operand boxes, MN-major operand boxes; io: 64 x 32 boxes for addend loads and
+  // result stores; tr: 32 x 64 boxes for the transposed stores
+  CUtensorMap x_k[2], x_mn[2], x_io[2], a_k, a_io, a_tr, b_k, b_io, b_tr;
   int2* tiles_sym = nullptr;
   int n_tiles_sym = 0;
   int2* tiles_full = nullptr;
@@ -516,27 +729,30 @@ TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1,
   pl->s = s; pl->l = l; pl->ldx = ldx; pl->lds = lds; pl->chunk = chunk;
   pl->X[0] = X0; pl->X[1] = X1; pl->A = A; pl->B = B;
   pl->n_sms = tc_num_sms();
-  pl->bn_sym = (s > 128) ? 256 : 128;
-  pl->bn_apply = (l > 128) ? 256 : 128;
+  pl->cg = (s > 128) ? 2 : 1;
   bool ok = true;
   for (int i = 0; i < 2; ++i) {
-    ok = ok && encode_map(&pl->x_k[i], pl->X[i], l, s, chunk, ldx, BK, 128);
-    ok = ok && encode_map(&pl->x_mn[i], pl->X[i], l, s, chunk, ldx, 64, BK);
+    ok = ok && encode_map(&pl->x_k[i], pl->X[i], l, s, chunk, ldx, BK, 128, true);
+    ok = ok && encode_map(&pl->x_mn[i], pl->X[i], l, s, chunk, ldx, 64, BK, true);
+    ok = ok && encode_map(&pl->x_io[i], pl->X[i], l, s, chunk, ldx, 64, 32, true);
   }
-  ok = ok && encode_map(&pl->a_k, A, s, s, chunk, lds, BK, 128);
-  ok = ok && encode_map(&pl->b_k, B, s, s, chunk, lds, BK, 128);
+  ok = ok && encode_map(&pl->a_k, A, s, s, chunk, lds, BK, 128, true);
+  ok = ok && encode_map(&pl->a_io, A, s, s, chunk, lds, 64, 32, true);
+  ok = ok && encode_map(&pl->a_tr, A, s, s, chunk, lds, 32, 64, false);
+  ok = ok && encode_map(&pl->b_k, B, s, s, chunk, lds, BK, 128, true);
+  ok = ok && encode_map(&pl->b_io, B, s, s, chunk, lds, 64, 32, true);
+  ok = ok && encode_map(&pl->b_tr, B, s, s, chunk, lds, 32, 64, false);
   if (!ok) {
     snprintf(err, errlen, "cuTensorMapEncodeTiled failed for shape %lld x %lld", (long long)s, (long long)l);
     delete pl;
     return nullptr;
   }
   std::vector<int2> sym, full;
-  const int tm_n = (int)((s + BM - 1) / BM);
-  const int tn_sym = (int)((s + pl->bn_sym - 1) / pl->bn_sym);
+  const int64_t T = 128 * pl->cg;
+  const int tm_n = (int)((s + T - 1) / T);
   for (int tm = 0; tm < tm_n; ++tm)
-    for (int tn = 0; tn < tn_sym; ++tn)
-      if ((int64_t)(tn + 1) * pl->bn_sym > (int64_t)tm * BM) sym.push_back(make_int2(tm, tn));
-  const int tn_full = (int)((l + pl->bn_apply - 1) / pl->bn_apply);
+    for (int tn = tm; tn < tm_n; ++tn) sym.push_back(make_int2(tm, tn));
+  const int tn_full = (int)((l + T - 1) / T);
   for (int tm = 0; tm < tm_n; ++tm)
     for (int tn = 0; tn < tn_full; ++tn) full.push_back(make_int2(tm, tn));
   pl->n_tiles_sym = (int)sym.size();
@@ -569,29 +785,21 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int kind, int n_mats, in
   p.scales = args.scales; p.mats = args.mats; p.sink_mode = args.sink_mode;
   p.s = pl->s; p.l = pl->l; p.status = args.status;
   p.M = (int)pl->s;
-  const int64_t sX = pl->s * pl->ldx, sS = pl->s * pl->lds;
-  __nv_bfloat16* Xin = reinterpret_cast<__nv_bfloat16*>(pl->X[xin]);
-  __nv_bfloat16* Xout = reinterpret_cast<__nv_bfloat16*>(pl->X[1 - xin]);
-  __nv_bfloat16* A = reinterpret_cast<__nv_bfloat16*>(pl->A);
-  __nv_bfloat16* B = reinterpret_cast<__nv_bfloat16*>(pl->B);
+  Maps5 m;
   if (kind == GEMM_GRAM) {
     p.N = (int)pl->s; p.Kd = (int)pl->l; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
-    p.D = A; p.ldd = pl->lds; p.strideD = sS;
-    return pl->bn_sym == 256 ? launch_one<256, false>(st, pl->x_k[xin], pl->x_k[xin], p, pl->n_sms)
-                             : launch_one<128, false>(st, pl->x_k[xin], pl->x_k[xin], p, pl->n_sms);
+    m = Maps5{&pl->x_k[xin], &pl->x_k[xin], &pl->a_io, &pl->a_io, &pl->a_tr};
+    return pl->cg == 2 ? launch_one<2, false>(st, m, p, pl->n_sms) : launch_one<1, false>(st, m, p, pl->n_sms);
   }
   if (kind == GEMM_POLY) {
     p.N = (int)pl->s; p.Kd = (int)pl->s; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
-    p.Cin = A; p.ldc = pl->lds; p.strideC = sS;
-    p.D = B; p.ldd = pl->lds; p.strideD = sS;
-    return pl->bn_sym == 256 ? launch_one<256, false>(st, pl->a_k, pl->a_k, p, pl->n_sms)
-                             : launch_one<128, false>(st, pl->a_k, pl->a_k, p, pl->n_sms);
+    m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, &pl->b_tr};
+    return pl->cg == 2 ? launch_one<2, false>(st, m, p, pl->n_sms) : launch_one<1, false>(st, m, p, pl->n_sms);
   }
   p.N = (int)pl->l; p.Kd = (int)pl->s; p.tiles = pl->tiles_full; p.n_tiles_per_mat = pl->n_tiles_full;
-  p.Cin = Xin; p.ldc = pl->ldx; p.strideC = sX;
-  p.D = (kind == GEMM_APPLY) ? Xout : nullptr; p.ldd = pl->ldx; p.strideD = sX;
-  return pl->bn_apply == 256 ? launch_one<256, true>(st, pl->b_k, pl->x_mn[xin], p, pl->n_sms)
-                             : launch_one<128, true>(st, pl->b_k, pl->x_mn[xin], p, pl->n_sms);
+  // FINAL stores nothing through tmD; the map still has to be a valid one
+  m = Maps5{&pl->b_k, &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin], &pl->x_io[1 - xin]};
+  return pl->cg == 2 ? launch_one<2, true>(st, m, p, pl->n_sms) : launch_one<1, true>(st, m, p, pl->n_sms);
 }
 
 }  // namespace muloco
