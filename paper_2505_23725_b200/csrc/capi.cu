@@ -259,12 +259,14 @@ muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_m
   return MULOCO_OK;
 }
 
-int pick_chunk(int64_t count, size_t per_slot, size_t budget, int n_sms) {
+// Matrices per workspace chunk: as many as the budget holds, then evened out so that
+// all chunks of a group have (nearly) the same size.
+int pick_chunk(int64_t count, size_t per_slot, size_t budget) {
   int64_t ch = (int64_t)(budget / (per_slot ? per_slot : 1));
   if (ch < 1) ch = 1;
-  if (ch > count) ch = count;
-  if (ch > n_sms && ch < count) ch = ch / n_sms * n_sms;
-  return (int)ch;
+  if (ch >= count) return (int)std::max<int64_t>(count, 1);
+  const int64_t n_chunks = (count + ch - 1) / ch;
+  return (int)((count + n_chunks - 1) / n_chunks);
 }
 
 muloco_status build_sync_tables(muloco_ctx* c) {
@@ -426,7 +428,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
   for (Group& g : c->groups) {
     const int np = prologue_partials_per_matrix(g.s, g.l);
     const size_t per_slot = make_layout(g.s, g.ldx, g.lds, 1, np, elt).total;
-    g.chunk = pick_chunk((int64_t)g.tensors.size() * K, per_slot, budget, c->n_sms);
+    g.chunk = pick_chunk((int64_t)g.tensors.size() * K, per_slot, budget);
     need = std::max(need, make_layout(g.s, g.ldx, g.lds, g.chunk, np, elt).total);
   }
   if (need) {
@@ -678,7 +680,7 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* c, const void* X, int3
   const int np = prologue_partials_per_matrix(s, l);
   const size_t per_slot = make_layout(s, ldx, lds, 1, np, elt).total;
   const size_t budget = c->cfg.workspace_bytes ? (size_t)c->cfg.workspace_bytes : ((size_t)6 << 30);
-  const int chunk = pick_chunk(batch, per_slot, budget, c->n_sms);
+  const int chunk = pick_chunk(batch, per_slot, budget);
   if (g.s != s || g.l != l || c->sa_mode != ns_mode || g.chunk != chunk || !c->sa_ws) {
     CK(cudaStreamSynchronize(c->st));
     destroy_group(g);

@@ -249,6 +249,14 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void prefetch_l2_bulk(const void* gptr, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
   asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -324,6 +332,24 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const int a_row = BM * (CG * tt.x + (int)rank);
       const int b_off = TM * tt.y + 128 * (int)rank;
       const uint32_t cta_bytes = A_STAGE_BYTES + (same ? 0u : B_STAGE_BYTES);
+      if (p.kind == GEMM_FINAL && p.sink_mode == SINK_UPDATE_W) {
+        // the parameters this CTA will update at the end of the tile: start moving them into L2 now
+        const MatDesc d = p.mats[mat];
+        const float* W = reinterpret_cast<const float*>(d.w);
+        const int c0 = TM * tt.y;
+        const int ncols = min(BN, p.N - c0), nrows = min(BM, p.M - a_row);
+        if (ncols > 0 && nrows > 0 && ((((uintptr_t)W) & 15) == 0)) {
+          if (!d.transposed) {
+            if ((p.l & 3) == 0 && (ncols & 3) == 0)
+              for (int r = lane; r < nrows; r += 32)
+                prefetch_l2_bulk(W + (int64_t)(a_row + r) * p.l + c0, (uint32_t)ncols * 4u);
+          } else {
+            if ((p.s & 3) == 0 && (nrows & 3) == 0)
+              for (int j = lane; j < ncols; j += 32)
+                prefetch_l2_bulk(W + (int64_t)(c0 + j) * p.s + a_row, (uint32_t)nrows * 4u);
+          }
+        }
+      }
       for (int kb = 0; kb < num_kb && alive; ++kb) {
         if (lane == 0) {
           if (mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, &abort_flag)) {
@@ -427,7 +453,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
     const bool has_cin = (p.kind != GEMM_GRAM);
     const bool stores = (p.kind != GEMM_FINAL);
-    uint32_t cin_issued = 0, cin_used = 0, st_count = 0;
+    uint32_t cin_issued = 0, cin_used = 0, st_count = 0, t_count = 0;
     int local_tile = 0;
     bool alive = true;
     for (int tile = unit; tile < total_tiles && alive; tile += n_units, ++local_tile) {
@@ -512,31 +538,57 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             for (int e = 0; e < 32; ++e) f[e] *= sc;
           }
           if (!stores) {
-            // ---- parameter update / output sink (fp32 tensor in its own layout) ----
+            // ---- parameter update / output sink (tensor in its own layout and type) ----
+            // Lanes run along the tensor's contiguous axis, so every access of the warp is one
+            // full line: for a tensor stored rows x cols as s x l that axis is the tile's column
+            // axis and the block is first turned through shared memory; for a tensor stored
+            // l x s it is the tile's row axis, which the lanes already hold.
             const int gjh = gj0 + h * 32;
-            if (row_ok && gjh < p.N) {
+            if (gjh < p.N) {
               const MatDesc d = p.mats[mat];
-              const bool full_chunk = (gjh + 32 <= p.N);
-              const bool fast = !d.transposed && p.sink_mode != SINK_STORE_BF16 && full_chunk &&
-                                ((p.l & 3) == 0) && ((((uintptr_t)d.w) & 15) == 0);
-              if (fast) {
-                float4* w4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(d.w) + (int64_t)gi * p.l + gjh);
-                if (p.sink_mode == SINK_UPDATE_W) {
-#pragma unroll
-                  for (int q = 0; q < 8; ++q) {
-                    float4 w = w4[q];
-                    w.x = fmaf(-d.lr_eff, f[q * 4 + 0], fmaf(-d.wd_term, w.x, w.x));
-                    w.y = fmaf(-d.lr_eff, f[q * 4 + 1], fmaf(-d.wd_term, w.y, w.y));
-                    w.z = fmaf(-d.lr_eff, f[q * 4 + 2], fmaf(-d.wd_term, w.z, w.z));
-                    w.w = fmaf(-d.lr_eff, f[q * 4 + 3], fmaf(-d.wd_term, w.w, w.w));
-                    w4[q] = w;
-                  }
-                } else {
+              const bool full = (gi0 + 32 <= p.M) && (gjh + 32 <= p.N);
+              if (full) {
+                float o[32];
+                int64_t base, stride;
+                if (!d.transposed) {
+                  const uint32_t tb = out_buf(t_count & 1u);
+                  ++t_count;
 #pragma unroll
                   for (int q = 0; q < 8; ++q)
-                    w4[q] = make_float4(f[q * 4 + 0], f[q * 4 + 1], f[q * 4 + 2], f[q * 4 + 3]);
+                    sts128(tb + (uint32_t)lane * 128u + ((uint32_t)(q ^ (lane & 7)) << 4),
+                           make_uint4(__float_as_uint(f[q * 4 + 0]), __float_as_uint(f[q * 4 + 1]),
+                                      __float_as_uint(f[q * 4 + 2]), __float_as_uint(f[q * 4 + 3])));
+                  __syncwarp();
+#pragma unroll
+                  for (int r = 0; r < 32; ++r)
+                    o[r] = __uint_as_float(lds32(tb + (uint32_t)r * 128u + ((uint32_t)((lane >> 2) ^ (r & 7)) << 4) +
+                                                 (uint32_t)(lane & 3) * 4u));
+                  base = (int64_t)gi0 * p.l + gjh + lane;
+                  stride = p.l;
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 32; ++e) o[e] = f[e];
+                  base = (int64_t)gjh * p.s + gi0 + lane;
+                  stride = p.s;
                 }
-              } else {
+                if (p.sink_mode == SINK_UPDATE_W) {
+                  float* W = reinterpret_cast<float*>(d.w) + base;
+                  float wv[32];
+#pragma unroll
+                  for (int r = 0; r < 32; ++r) wv[r] = W[(int64_t)r * stride];
+#pragma unroll
+                  for (int r = 0; r < 32; ++r)
+                    W[(int64_t)r * stride] = fmaf(-d.lr_eff, o[r], fmaf(-d.wd_term, wv[r], wv[r]));
+                } else if (p.sink_mode == SINK_STORE_F32) {
+                  float* O = reinterpret_cast<float*>(d.w) + base;
+#pragma unroll
+                  for (int r = 0; r < 32; ++r) O[(int64_t)r * stride] = o[r];
+                } else {
+                  __nv_bfloat16* O = reinterpret_cast<__nv_bfloat16*>(d.w) + base;
+#pragma unroll
+                  for (int r = 0; r < 32; ++r) O[(int64_t)r * stride] = __float2bfloat16_rn(o[r]);
+                }
+              } else if (row_ok) {
 #pragma unroll
                 for (int e = 0; e < 32; ++e)
                   if (gjh + e < p.N) sink_element(d, p.sink_mode, p.s, p.l, gi, gjh + e, f[e]);
@@ -590,7 +642,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         mbar_arrive_cluster(CG == 2 ? map_to_rank(te, 0) : te);
       }
     }
-    if (lane == 0) bulk_wait_all();
+    bulk_wait_all();
   }
 
   // ------------------------------- teardown ----------------------------------
