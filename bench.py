@@ -203,9 +203,17 @@ def main():
     ap.add_argument("--workspace-gb", type=float, default=0.0)
     ap.add_argument("--ns-only", type=int, nargs=3, metavar=("BATCH", "ROWS", "COLS"), default=None,
                     help="kernel study: time muloco_newton_schulz (bf16 engine) on a batch of one shape")
+    ap.add_argument("--sync-only", type=int, nargs=3, metavar=("K", "MPARAMS", "QUANT"), default=None,
+                    help="kernel study: time muloco_outer_sync on MPARAMS million parameters, K replicas, "
+                         "QUANT in {0, 4, 8}")
+    ap.add_argument("--adamw-only", type=int, nargs=2, metavar=("K", "MPARAMS"), default=None,
+                    help="kernel study: time the AdamW part of muloco_inner_step on MPARAMS million parameters")
     args = ap.parse_args()
     if args.ns_only:
         run_ns_only(args)
+        return
+    if args.sync_only or args.adamw_only:
+        run_elementwise_only(args)
         return
 
     from paper_2505_23725_b200 import configs
@@ -366,6 +374,53 @@ def run_ns_only(args):
                       "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
                       "frac_of_burst_peak": tf / peaks["bf16_tflops"], "prologue_ms": ph["prologue"] / args.steps,
                       "launches": int(launches)}))
+    opt.close()
+
+
+def run_elementwise_only(args):
+    """Small cases for kernel studies and ncu captures of the two streaming kernels: the
+    outer synchronisation (--sync-only) or AdamW (--adamw-only) over a few large tensors."""
+    import torch
+    from paper_2505_23725_b200 import binding, configs
+    import __graft_entry__ as entry
+    entry.build()
+    sync = args.sync_only is not None
+    K, mparams = (args.sync_only[0], args.sync_only[1]) if sync else args.adamw_only
+    quant = args.sync_only[2] if sync else 0
+    rows = max(1, mparams * 1000000 // (8 * 4096))
+    ts = [configs.Tensor(f"t{i}", rows, 4096, configs.ADAMW, 0) for i in range(8)]
+    w = configs.Workload("elementwise-only", K=K, H=1, J=1, tensors=ts, muon_lr=0.02, muon_beta=0.9, muon_wd=0.01,
+                         outer_lr=0.7, outer_momentum=0.9, quant_bits=quant)
+    opt = binding.MuLoCo(w, "cuda:0", init_seed=1, alloc_grads=not sync)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(0)
+    if sync:
+        for k in range(K):
+            opt.flat_theta_k[k].normal_(0.0, 0.02, generator=gen)
+    else:
+        for k in range(K):
+            opt.flat_grads[k].normal_(0.0, 0.01, generator=gen)
+    call = (lambda: opt.outer_sync(-1)) if sync else (lambda: opt.inner_step(-1, None, 1.0))
+    for _ in range(args.warmup):
+        call()
+    opt.set_timing(True); opt.get_timings()
+    torch.cuda.synchronize()
+    torch.cuda.cudart().cudaProfilerStart()
+    for _ in range(args.steps):
+        call()
+    ph, launches = opt.get_timings()
+    torch.cuda.cudart().cudaProfilerStop()
+    opt.sync_status()
+    peaks = load_peaks()
+    n = w.n_params
+    if sync:
+        ms = ph["sync"] / args.steps
+        nbytes = n * (8.0 * K + 16.0)
+    else:
+        ms = ph["adamw"] / args.steps
+        nbytes = n * K * 28.0
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    print(json.dumps({"sync_only" if sync else "adamw_only": [K, mparams, quant], "params": n, "ms_per_call": ms,
+                      "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "launches": int(launches)}))
     opt.close()
 
 

@@ -18,7 +18,7 @@ import numpy as np
 from . import configs as _cfg
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmuloco.so")
+LIB_PATH = os.environ.get("MULOCO_LIBRARY", os.path.join(_HERE, "libmuloco.so"))
 
 OK, EINVAL, ESHAPE, ENOMEM, ECUDA, ENONFINITE, ETIMEOUT, ESTATE = range(8)
 STATUS_NAMES = ["OK", "EINVAL", "ESHAPE", "ENOMEM", "ECUDA", "ENONFINITE", "ETIMEOUT", "ESTATE"]

@@ -28,17 +28,18 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+def build_library(force: bool = False, verbose: bool = False, lib_path: str = LIB) -> str:
     """Compile every CUDA source of the package for sm_100a into one shared library."""
-    if not force and not needs_build():
+    if not force and lib_path == LIB and not needs_build():
         return LIB
     objs = []
-    bdir = os.path.join(HERE, "_build")
+    bdir = os.path.join(HERE, "_build") if lib_path == LIB else lib_path + ".objs"
     os.makedirs(bdir, exist_ok=True)
     common = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
     if verbose:
         common += ["-Xptxas", "-v"]
+    common += os.environ.get("MULOCO_NVCC_FLAGS", "").split()   # extra -D... for tuning studies
     procs = []
     for src in SOURCES:
         obj = os.path.join(bdir, src.replace(".cu", ".o"))
@@ -51,8 +52,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}")
-    subprocess.check_call([_nvcc(), "-shared", "-o", LIB] + objs)
-    return LIB
+    subprocess.check_call([_nvcc(), "-shared", "-o", lib_path] + objs)
+    return lib_path
 
 
 if __name__ == "__main__":

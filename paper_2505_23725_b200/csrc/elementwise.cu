@@ -26,6 +26,15 @@ __device__ __forceinline__ float to_x<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ __nv_bfloat16 to_x<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+__device__ __forceinline__ void store_x4(float* p, float4 u) { *reinterpret_cast<float4*>(p) = u; }
+__device__ __forceinline__ void store_x4(__nv_bfloat16* p, float4 u) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(u.x, u.y), hi = __floats2bfloat162_rn(u.z, u.w);
+  uint2 v;
+  v.x = *reinterpret_cast<uint32_t*>(&lo);
+  v.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = v;
+}
+
 // One CTA = one 32 x 128 tile of X (s x l view) of one matrix.
 // The value that enters the sum of squares is the fp32 U (before bf16 rounding).
 template <typename XT>
@@ -37,7 +46,12 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   __shared__ float red[PRO_THREADS / 32];
   const int mat = blockIdx.y;
   const MatDesc d = mats[mat];
-  const int ti = blockIdx.x / tiles_j, tj = blockIdx.x % tiles_j;
+  // Tile order follows the tensor's own memory order, so that the CTAs resident at one
+  // time read neighbouring addresses: tj fastest for a tensor stored s x l, ti fastest for
+  // one stored l x s (its rows are the j axis).
+  const int tiles_i = n_part / tiles_j;
+  const int ti = d.transposed ? (int)(blockIdx.x % tiles_i) : (int)(blockIdx.x / tiles_j);
+  const int tj = d.transposed ? (int)(blockIdx.x / tiles_i) : (int)(blockIdx.x % tiles_j);
   const int64_t i0 = (int64_t)ti * PRO_TI, j0 = (int64_t)tj * PRO_TJ;
   XT* Xm = X + (int64_t)mat * s * ldx;
   float ss = 0.f;
@@ -58,7 +72,57 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
     return u;
   };
 
-  if (!d.transposed) {
+  const bool vec4 = !d.transposed && ((l & 3) == 0) && ((ldx & 3) == 0) &&
+                    ((((uintptr_t)d.g | (uintptr_t)d.m) & 15) == 0) && ((((uintptr_t)Xm) & 15) == 0);
+  if (vec4) {
+    // tensor is s x l with 16-byte aligned rows: four consecutive j per thread.  All loads of
+    // the thread's four rows are issued before the first store (the stores to m would
+    // otherwise order the later loads behind them).
+    const int tx = tid & 31, ty = tid >> 5;   // 32 x 8
+    constexpr int R = PRO_TI / 8;
+    const int64_t j = j0 + tx * 4;
+    const bool src_bf16 = (src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16);
+    float4 g[R], mo[R];
+    bool ok[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int64_t i = i0 + ty + r * 8;
+      ok[r] = (i < s) && (j < l);
+      g[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      mo[r] = g[r];
+      if (!ok[r]) continue;
+      const int64_t idx = i * l + j;
+      if (src_bf16) {
+        const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(d.g) + idx));
+        g[r] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+      } else {
+        g[r] = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(d.g) + idx));
+      }
+      if (src_mode == SRC_MUON) mo[r] = *reinterpret_cast<const float4*>(d.m + idx);
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (!ok[r]) continue;
+      const int64_t i = i0 + ty + r * 8;
+      const int64_t idx = i * l + j;
+      float4 u = g[r];
+      if (src_mode == SRC_MUON) {
+        float4 mn;
+        mn.x = fmaf(beta, mo[r].x, g[r].x); mn.y = fmaf(beta, mo[r].y, g[r].y);
+        mn.z = fmaf(beta, mo[r].z, g[r].z); mn.w = fmaf(beta, mo[r].w, g[r].w);
+        *reinterpret_cast<float4*>(d.m + idx) = mn;
+        if (nesterov) {
+          u.x = fmaf(beta, mn.x, g[r].x); u.y = fmaf(beta, mn.y, g[r].y);
+          u.z = fmaf(beta, mn.z, g[r].z); u.w = fmaf(beta, mn.w, g[r].w);
+        } else {
+          u = mn;
+        }
+      }
+      ss = fmaf(u.x, u.x, ss); ss = fmaf(u.y, u.y, ss); ss = fmaf(u.z, u.z, ss); ss = fmaf(u.w, u.w, ss);
+      store_x4(Xm + i * ldx + j, u);
+    }
+  } else if (!d.transposed) {
     // tensor is s x l: X[i][j] = T[i][j]; lanes run along j
     const int tx = tid & 31, ty = tid >> 5;   // 32 x 8
 #pragma unroll
@@ -78,16 +142,43 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   } else {
     // tensor is l x s: X[i][j] = T[j][i]; read with lanes along i, write with lanes along j
     const int tx = tid & 31, ty = tid >> 5;
-#pragma unroll 4
-    for (int r = 0; r < PRO_TJ / 8; ++r) {
-      const int jj = ty + r * 8;
-      const int64_t j = j0 + jj, i = i0 + tx;
-      float u = 0.f;
-      if (j < l && i < s) {
-        u = produce(j * s + i);
-        ss = fmaf(u, u, ss);
+    const int64_t i = i0 + tx;
+    constexpr int RB = 8;   // rows per batch: their loads are all issued before the first store
+#pragma unroll 1
+    for (int rb = 0; rb < PRO_TJ / 8; rb += RB) {
+      float gv[RB], mv[RB];
+      bool ok[RB];
+#pragma unroll
+      for (int q = 0; q < RB; ++q) {
+        const int64_t j = j0 + ty + (rb + q) * 8;
+        ok[q] = (j < l) && (i < s);
+        gv[q] = 0.f; mv[q] = 0.f;
+        if (!ok[q]) continue;
+        const int64_t idx = j * s + i;
+        if (src_mode == SRC_MUON) {
+          gv[q] = load_g(d.g, idx, g_is_bf16);
+          mv[q] = d.m[idx];
+        } else if (src_mode == SRC_RAW_F32) {
+          gv[q] = reinterpret_cast<const float*>(d.g)[idx];
+        } else {
+          gv[q] = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(d.g)[idx]);
+        }
       }
-      tile[jj][tx] = u;
+#pragma unroll
+      for (int q = 0; q < RB; ++q) {
+        const int jj = ty + (rb + q) * 8;
+        float u = 0.f;
+        if (ok[q]) {
+          u = gv[q];
+          if (src_mode == SRC_MUON) {
+            const float mn = fmaf(beta, mv[q], gv[q]);
+            d.m[(j0 + jj) * s + i] = mn;
+            u = nesterov ? fmaf(beta, mn, gv[q]) : mn;
+          }
+          ss = fmaf(u, u, ss);
+        }
+        tile[jj][tx] = u;
+      }
     }
     __syncthreads();
 #pragma unroll
@@ -241,7 +332,8 @@ void launch_finalize_scales(cudaStream_t st, const float* partials, int n_part, 
 void launch_adamw(cudaStream_t st, const AdamSeg* segs, int n_segs, int64_t n_units, int g_is_bf16,
                   float beta1, float beta2, float eps) {
   if (n_units <= 0 || n_segs <= 0) return;
-  int64_t blocks = n_units < (int64_t)148 * 16 ? n_units : (int64_t)148 * 16;
+  // one unit per CTA, launched in address order (the resident CTAs then share DRAM pages)
+  int64_t blocks = n_units < 0x7fffffffLL ? n_units : 0x7fffffffLL;
   adamw_kernel<<<(unsigned)blocks, ADAM_THREADS, 0, st>>>(segs, n_segs, n_units, g_is_bf16, beta1,
                                                           beta2, eps);
 }

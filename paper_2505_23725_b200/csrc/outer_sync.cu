@@ -5,8 +5,8 @@
 //
 // Work unit = one block of `block` (<= 128) consecutive elements of one row,
 // handled by one warp, four elements per lane (128-bit accesses when the row
-// pitch allows).  A CTA owns a contiguous span of units so that each of the
-// K+2 streams is read in long runs.
+// pitch allows).  A CTA owns a short contiguous span of units; CTAs are launched
+// in address order.
 #include <float.h>
 
 #include "internal.h"
@@ -17,6 +17,10 @@ namespace {
 
 constexpr int SYNC_THREADS = 256;
 constexpr int SYNC_WARPS = SYNC_THREADS / 32;
+// Units per warp.  Small CTAs in launch order: the CTAs resident at any moment then work on
+// one narrow window of each of the K+2 streams, which keeps DRAM pages open (measured: 6.56 TB/s
+// with 4 units per warp against 5.8 TB/s with a few long spans per SM).
+constexpr int SYNC_UNITS_PER_WARP = 4;
 
 __device__ __forceinline__ int find_seg(const SyncSeg* __restrict__ segs, int n, int64_t unit) {
   int lo = 0, hi = n - 1;
@@ -266,14 +270,10 @@ void launch_sync_q(cudaStream_t st, dim3 grid, const SyncSeg* segs, int n_segs, 
 void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
                        int K, int64_t n_units, int block, int quant_bits, float outer_lr, float mu,
                        int* status, int n_sms) {
+  (void)n_sms;
   if (n_units <= 0) return;
-  // persistent-style grid: a multiple of the SM count, each CTA a contiguous span
-  int64_t ctas = (int64_t)n_sms * 8;
-  int64_t min_units = SYNC_WARPS * 4;   // at least a few units per warp
-  if (ctas * min_units > n_units) ctas = (n_units + min_units - 1) / min_units;
-  if (ctas < 1) ctas = 1;
-  const int64_t upc = (n_units + ctas - 1) / ctas;
-  ctas = (n_units + upc - 1) / upc;
+  const int64_t upc = (int64_t)SYNC_WARPS * SYNC_UNITS_PER_WARP;
+  const int64_t ctas = (n_units + upc - 1) / upc;
   const float inv_k = 1.0f / (float)K;
   dim3 grid((unsigned)ctas);
   if (quant_bits == 8)
