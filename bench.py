@@ -208,7 +208,13 @@ def main():
                          "QUANT in {0, 4, 8}")
     ap.add_argument("--adamw-only", type=int, nargs=2, metavar=("K", "MPARAMS"), default=None,
                     help="kernel study: time the AdamW part of muloco_inner_step on MPARAMS million parameters")
+    ap.add_argument("--muon-only", type=int, nargs=4, metavar=("K", "LAYERS", "D", "F"), default=None,
+                    help="kernel study: muloco_inner_step on LAYERS layers of hidden matrices only "
+                         "(prologue + Newton-Schulz with the fused parameter update), K workers")
     args = ap.parse_args()
+    if args.muon_only:
+        run_muon_only(args)
+        return
     if args.ns_only:
         run_ns_only(args)
         return
@@ -374,6 +380,37 @@ def run_ns_only(args):
                       "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
                       "frac_of_burst_peak": tf / peaks["bf16_tflops"], "prologue_ms": ph["prologue"] / args.steps,
                       "launches": int(launches)}))
+    opt.close()
+
+
+def run_muon_only(args):
+    """Small case of the real inner step for ncu captures: hidden matrices only, so the
+    launches are exactly those of the benchmark's Muon path at a fraction of its depth."""
+    import torch
+    from paper_2505_23725_b200 import binding, configs, synth
+    import __graft_entry__ as entry
+    entry.build()
+    K, L, d, F = args.muon_only
+    w = configs.mini_workload(K=K, H=1, J=1, ns_mode="bf16", L=L, d=d, F=F, muon_lr=4.42e-2, muon_beta=0.9,
+                              muon_wd=6.25e-4)
+    opt = binding.MuLoCo(w, "cuda:0", init_seed=1, alloc_grads=True,
+                         workspace_bytes=int(args.workspace_gb * (1 << 30)))
+    synth.torch_fill_gradients(opt.grads, w.tensors, w.K, 3, opt.device)
+    for _ in range(args.warmup):
+        opt.inner_step(-1, None, 1.0)
+    opt.set_timing(True); opt.get_timings()
+    torch.cuda.synchronize()
+    torch.cuda.cudart().cudaProfilerStart()
+    for _ in range(args.steps):
+        opt.inner_step(-1, None, 1.0)
+    ph, launches = opt.get_timings()
+    torch.cuda.cudart().cudaProfilerStop()
+    opt.sync_status()
+    peaks = load_peaks()
+    tf = w.ns_flops_credited() / (ph["ns"] / args.steps * 1e-3) / 1e12
+    print(json.dumps({"muon_only": [K, L, d, F], "params_per_replica": w.n_params, "ns_ms": ph["ns"] / args.steps,
+                      "prologue_ms": ph["prologue"] / args.steps, "ns_tflops_credited": tf,
+                      "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"], "launches": int(launches)}))
     opt.close()
 
 
