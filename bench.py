@@ -31,9 +31,12 @@ if ROOT not in sys.path:
 METRIC = "optimizer-step params/sec (inner Muon + outer sync) at K workers"
 UNIT = "param-updates/s"
 
-# DRAM traffic (bytes) per credited FLOP of the Newton-Schulz GEMM kernels, from the
-# ncu capture summarised in profiles/; None until a capture exists.
-NS_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM traffic of the Newton-Schulz GEMM launches per hidden-matrix parameter, worker and inner
+# step, from the ncu capture summarised in profiles/ns_tc_kernel_muon-only_K16_L2_d1024_F2816.md
+# (24.33 GB over the 30 launches of a 2-layer, K=16 inner step with 25,690,112 parameters per
+# replica).  It grows in proportion to the number of matrices, so it is scaled by the parameter
+# count; it holds for the d=1024, F=2816 shape mix only.
+NS_TRAFFIC_BYTES_PER_PARAM = {(1024, 2816): 24.334e9 / (25690112 * 16)}
 
 
 def load_peaks():
@@ -304,10 +307,19 @@ def main():
     ns_ms_per_inner = phases["ns"] / inner_steps
     ns_tflops = w.ns_flops_credited() / (ns_ms_per_inner * 1e-3) / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
-    ns_launches_per_inner = None
+    ns_launches_per_inner = phases_launches_ns(w, opt)
+    shape_key = None
+    for tn in w.tensors:
+        if tn.name.endswith(".w1"):
+            shape_key = (tn.rows, tn.cols)
+            break
+    per_param = NS_TRAFFIC_BYTES_PER_PARAM.get(shape_key)
+    traffic = (per_param * w.n_muon_params * w.K / ns_launches_per_inner) if per_param else None
     roofline = {"bound": "tensor", "kernel": "ns_tc_kernel (Gram / polynomial / apply GEMMs of Newton-Schulz)",
                 "achieved": ns_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": ns_tflops / peak_tf,
-                "peak_source": f"{peaks['source']} sustained bf16 matmul", "traffic": NS_TRAFFIC_BYTES_PER_LAUNCH,
+                "peak_source": f"{peaks['source']} sustained bf16 matmul (kernel timed inside a long step)",
+                "launches_per_inner_step": ns_launches_per_inner,
+                "traffic": traffic, "traffic_unit": "bytes per launch (average over the launches of an inner step)",
                 "flops_convention": "credited 5*(4 s^2 l + 2 s^3) per matrix; symmetric products run upper-triangle tiles only",
                 "ms_per_inner_step": ns_ms_per_inner}
     n_sync_rounds = args.steps
@@ -346,6 +358,23 @@ def main():
     if distributed:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def phases_launches_ns(w, opt):
+    """Newton-Schulz GEMM launches per inner step: 15 per chunk of every shape group."""
+    ph, n = 0, 0
+    groups = {}
+    for t in w.tensors:
+        if t.kind == "muon":
+            key = (min(t.rows, t.cols), max(t.rows, t.cols))
+            groups[key] = groups.get(key, 0) + w.K
+    budget = opt.cfg.workspace_bytes or (6 << 30)
+    for (s_, l_), count in groups.items():
+        ldx, lds = (l_ + 7) // 8 * 8, (s_ + 7) // 8 * 8
+        per = 2 * s_ * ldx * 2 + 2 * s_ * lds * 2
+        ch = max(1, min(count, budget // per))
+        n += 15 * ((count + ch - 1) // ch)
+    return n
 
 
 def run_ns_only(args):
