@@ -99,6 +99,26 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def rank_seeds(base_seed: int, rank: int):
+    """Seeds of rank `rank`'s independent K-worker problem: (initial weights, gradients)."""
+    return base_seed + 1000 * rank, base_seed + 17 * rank
+
+
+def max_over_ranks(ms: float, dist=None, device="cpu") -> float:
+    """Device time of the slowest rank (every rank gets the same number back)."""
+    if dist is None:
+        return float(ms)
+    import torch
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_value(world: int, units_per_rank: float, ms_per_step: float) -> float:
+    """Units all ranks processed per second: every rank runs its own full problem (weak scaling)."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 def oracle_cores():
     try:
         from threadpoolctl import threadpool_info
@@ -251,9 +271,10 @@ def main():
     dev = f"cuda:{local_rank}"
     torch.cuda.set_device(dev)
 
-    opt = binding.MuLoCo(w, dev, init_seed=w.seed + 1000 * rank, alloc_grads=True,
+    seed_init, seed_grad = rank_seeds(w.seed, rank)
+    opt = binding.MuLoCo(w, dev, init_seed=seed_init, alloc_grads=True,
                          workspace_bytes=int(args.workspace_gb * (1 << 30)))
-    synth.torch_fill_gradients(opt.grads, w.tensors, w.K, w.seed + 17 * rank, opt.device)
+    synth.torch_fill_gradients(opt.grads, w.tensors, w.K, seed_grad, opt.device)
     torch.cuda.synchronize()
 
     def one_round(t0):
@@ -293,13 +314,10 @@ def main():
     phases, launches = opt.get_timings()
     opt.set_timing(False)
     opt.sync_status()
-    if distributed:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, dist if distributed else None, dev)
     ms_per_step = ms_total / args.steps
     units_per_round = w.K * w.n_params * w.H
-    value = world * units_per_round / (ms_per_step * 1e-3)
+    value = whole_job_value(world, units_per_round, ms_per_step)
 
     # ---- roofline of the dominant kernel (Newton-Schulz tensor-core GEMMs) ----------------
     peaks = load_peaks()
@@ -526,13 +544,10 @@ def run_e2e(opt, w, torch, dist, world):
     e1.record(opt.stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
-    if dist:
-        tt = torch.tensor([ms], device=opt.device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = max_over_ranks(ms, dist, opt.device)
     opt.sync_status()
     h2d = w.n_params * elt * w.K * w.H
-    return {"value": world * w.K * w.n_params * w.H / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": whole_job_value(world, w.K * w.n_params * w.H, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "rounds_timed": 1, "host_grad_sets": n_sets}
 
 
