@@ -103,6 +103,8 @@ struct muloco_ctx {
   // per-call tables
   MatDesc* d_mats = nullptr;
   AdamSeg* d_adam = nullptr;
+  char* d_wmaps = nullptr;                 // [K][n] TMA descriptors over theta_k (bf16 engine only)
+  std::vector<char> wmap_ok;               // [K][n]
   char* h_ring[RING] = {nullptr, nullptr, nullptr};
   cudaEvent_t ring_ev[RING];
   bool ring_used[RING] = {false, false, false};
@@ -455,6 +457,21 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
     CKC(cudaEventCreateWithFlags(&c->ring_ev[r], cudaEventDisableTiming));
   }
 
+  if (cfg->ns_mode == MULOCO_NS_BF16 && !c->muon_ids.empty()) {
+    // one TMA descriptor per (worker, hidden matrix) for the fused parameter update
+    std::vector<char> hmaps((size_t)K * n_tensors * TC_MAP_BYTES, 0);
+    c->wmap_ok.assign((size_t)K * n_tensors, 0);
+    for (int k = 0; k < K; ++k)
+      for (int i : c->muon_ids) {
+        const TensorInfo& t = c->T[i];
+        const size_t e = (size_t)k * n_tensors + i;
+        c->wmap_ok[e] = tc_encode_w_map(hmaps.data() + e * TC_MAP_BYTES, t.theta_k[k], t.rows, t.cols,
+                                        t.rows > t.cols) ? 1 : 0;
+      }
+    CKC(cudaMalloc(&c->d_wmaps, hmaps.size()));
+    CKC(cudaMemcpy(c->d_wmaps, hmaps.data(), hmaps.size(), cudaMemcpyHostToDevice));
+  }
+
   if (build_sync_tables(c) != MULOCO_OK) return bail(MULOCO_ECUDA);
 
   // Algorithm 1, line 2: u <- 0, inner state <- 0, theta_k <- theta_g
@@ -485,6 +502,7 @@ MULOCO_API void muloco_destroy(muloco_ctx* c) {
   if (c->d_replicas) cudaFree(c->d_replicas);
   if (c->d_mats) cudaFree(c->d_mats);
   if (c->d_adam) cudaFree(c->d_adam);
+  if (c->d_wmaps) cudaFree(c->d_wmaps);
   if (c->stage) cudaFree(c->stage);
   for (FragTable& f : c->frags)
     if (f.d_segs) cudaFree(f.d_segs);
@@ -534,6 +552,8 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
         d.wd_term = (float)((f.wd_uses_scaled_lr ? eta : lr) * (double)f.muon_wd * (double)t.wd_mult);
         d.transposed = t.rows > t.cols;
         d.pad = 0;
+        const size_t e = (size_t)k * n + i;
+        d.wmap = (c->d_wmaps && c->wmap_ok[e]) ? c->d_wmaps + e * TC_MAP_BYTES : nullptr;
         hm[nm++] = d;
       }
   }
@@ -716,6 +736,7 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* c, const void* X, int3
       d.lr_eff = 0.f; d.wd_term = 0.f;
       d.transposed = rows > cols;
       d.pad = 0;
+      d.wmap = nullptr;
       hm[j] = d;
     }
     // pageable source: the copy is staged before the call returns, so hm may be reused

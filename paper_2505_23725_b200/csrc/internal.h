@@ -24,6 +24,8 @@ struct MatDesc {
   float wd_term;   // eta_wd * lambda * wd_mult (multiplies W)
   int32_t transposed;  // 1: tensor is l x s (rows > cols)
   int32_t pad;
+  const void* wmap;    // device address of a 128-byte TMA descriptor over W (32 x 32 fp32 boxes) for the
+                       // fused parameter update of the tensor-core engine, or NULL (plain accesses)
 };
 
 enum SrcMode : int { SRC_MUON = 0, SRC_RAW_F32 = 1, SRC_RAW_BF16 = 2 };
@@ -62,6 +64,11 @@ void tc_plan_destroy(TcGroupPlan*);
 cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* plan, int kind, int n_mats, int xin,
                       const NsIterArgs& args);
 int tc_num_sms();
+// Encodes (into 128 bytes at `out_host`) the TMA descriptor of a rows x cols fp32 tensor for 32 x 32
+// boxes; swizzled for tensors stored s x l, plain for tensors stored l x s.  False when the tensor
+// cannot be addressed by TMA (base not 16-byte aligned or cols not a multiple of 4).
+bool tc_encode_w_map(void* out_host, void* base, int64_t rows, int64_t cols, int transposed);
+constexpr size_t TC_MAP_BYTES = 128;
 
 // AdamW: one entry per (worker, tensor).
 struct AdamSeg {

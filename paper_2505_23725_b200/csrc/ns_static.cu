@@ -107,6 +107,7 @@ extern "C" MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, 
     hm[j].lr_eff = 0.f; hm[j].wd_term = 0.f;
     hm[j].transposed = rows > cols;
     hm[j].pad = 0;
+    hm[j].wmap = nullptr;
   }
   MatDesc* d_mats = reinterpret_cast<MatDesc*>(base + o_mats);
   int* d_status = reinterpret_cast<int*>(base + o_status);

@@ -155,6 +155,20 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
                : "memory");
 }
+// 2-D forms, descriptor in global memory (the per-matrix maps of the parameter tensors)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const void* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_2() { asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory"); }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -254,9 +268,6 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ void prefetch_l2_bulk(const void* gptr, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
   asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -282,6 +293,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t bar_tfull[2];
   __shared__ __align__(8) uint64_t bar_tempty[2];       // used in the CTA of rank 0
   __shared__ __align__(8) uint64_t bar_cin[4][2];
+  __shared__ __align__(8) uint64_t bar_w[4][4];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile int abort_flag;
 
@@ -310,8 +322,10 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       mbar_init(smem_u32(&bar_tfull[a]), 1);
       mbar_init(smem_u32(&bar_tempty[a]), 4 * CG);
     }
-    for (int w = 0; w < 4; ++w)
+    for (int w = 0; w < 4; ++w) {
       for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bar_cin[w][b]), 1);
+      for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&bar_w[w][b]), 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -332,24 +346,6 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const int a_row = BM * (CG * tt.x + (int)rank);
       const int b_off = TM * tt.y + 128 * (int)rank;
       const uint32_t cta_bytes = A_STAGE_BYTES + (same ? 0u : B_STAGE_BYTES);
-      if (p.kind == GEMM_FINAL && p.sink_mode == SINK_UPDATE_W) {
-        // the parameters this CTA will update at the end of the tile: start moving them into L2 now
-        const MatDesc d = p.mats[mat];
-        const float* W = reinterpret_cast<const float*>(d.w);
-        const int c0 = TM * tt.y;
-        const int ncols = min(BN, p.N - c0), nrows = min(BM, p.M - a_row);
-        if (ncols > 0 && nrows > 0 && ((((uintptr_t)W) & 15) == 0)) {
-          if (!d.transposed) {
-            if ((p.l & 3) == 0 && (ncols & 3) == 0)
-              for (int r = lane; r < nrows; r += 32)
-                prefetch_l2_bulk(W + (int64_t)(a_row + r) * p.l + c0, (uint32_t)ncols * 4u);
-          } else {
-            if ((p.s & 3) == 0 && (nrows & 3) == 0)
-              for (int j = lane; j < ncols; j += 32)
-                prefetch_l2_bulk(W + (int64_t)(c0 + j) * p.s + a_row, (uint32_t)nrows * 4u);
-          }
-        }
-      }
       for (int kb = 0; kb < num_kb && alive; ++kb) {
         if (lane == 0) {
           if (mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, &abort_flag)) {
@@ -453,6 +449,13 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
     const bool has_cin = (p.kind != GEMM_GRAM);
     const bool stores = (p.kind != GEMM_FINAL);
+    // parameter update through TMA: a ring of four 32 x 32 fp32 blocks in the staging space that
+    // the direct and mirrored results use in the other products
+    auto w_buf = [&](uint32_t b) { return epi + (2u + b) * EPI_BLOCK_BYTES; };
+    const uint32_t w_bar0 = smem_u32(&bar_w[ew][0]);
+    auto w_bar = [&](uint32_t b) { return w_bar0 + b * 8u; };
+    const bool upd = (p.kind == GEMM_FINAL && p.sink_mode == SINK_UPDATE_W);
+    uint32_t w_issued = 0, w_used = 0;
     uint32_t cin_issued = 0, cin_used = 0, st_count = 0, t_count = 0;
     int local_tile = 0;
     bool alive = true;
@@ -483,6 +486,32 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         ++cin_issued;
       };
       if (has_cin && todo) issue_cin(__ffs(todo) - 1);
+      // fused parameter update: the old parameters come in as 32 x 32 blocks, two steps ahead
+      MatDesc dsc;
+      dsc.wmap = nullptr; dsc.transposed = 0; dsc.lr_eff = 0.f; dsc.wd_term = 0.f;
+      if (upd) dsc = p.mats[mat];
+      const bool use_tma = upd && dsc.wmap != nullptr && todo != 0;
+      int n_hb = 0;                                      // 32-column blocks of this warp in this tile
+      if (use_tma) n_hb = min(2 * NCH, (p.N - TM * tt.y + 31) >> 5);
+      auto issue_w = [&](int hb) {
+        if (lane == 0) {
+          const uint32_t b = w_issued & 3u;
+          const int gjh = TM * tt.y + hb * 32;
+          mbar_expect_tx(w_bar(b), EPI_BLOCK_BYTES);
+          if (!dsc.transposed) tma_load_2d(w_buf(b), dsc.wmap, w_bar(b), gjh, gi0);
+          else tma_load_2d(w_buf(b), dsc.wmap, w_bar(b), gi0, gjh);
+        }
+        ++w_issued;
+      };
+      if (use_tma) {
+        if (lane == 0) bulk_wait_read_2();               // blocks stored three and more steps ago have left the ring
+        __syncwarp();
+        issue_w(0);
+        if (n_hb > 1) issue_w(1);
+      } else if (upd) {
+        if (lane == 0) bulk_wait_read_0();               // plain path reuses the staging space
+        __syncwarp();
+      }
       if (!mbar_wait(smem_u32(&bar_tfull[acc]), acc_phase, &abort_flag)) alive = false;
       alive = __all_sync(0xffffffffu, alive);
       if (!alive) break;
@@ -544,7 +573,50 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             // axis and the block is first turned through shared memory; for a tensor stored
             // l x s it is the tile's row axis, which the lanes already hold.
             const int gjh = gj0 + h * 32;
-            if (gjh < p.N) {
+            if (use_tma) {
+              if (gjh < p.N) {
+                const int hb = 2 * c + h;
+                if (lane == 0) bulk_wait_read_1();       // the block stored two steps ago has left the ring
+                __syncwarp();
+                if (hb + 2 < n_hb) issue_w(hb + 2);
+                bool ok = mbar_wait(w_bar(w_used & 3u), (w_used >> 2) & 1u, &abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { alive = false; break; }
+                const uint32_t wb = w_buf(w_used & 3u);
+                if (!dsc.transposed) {
+                  // block rows are tile rows: each lane owns one 128-byte row (swizzled)
+#pragma unroll
+                  for (int q = 0; q < 8; ++q) {
+                    const uint32_t ad = wb + (uint32_t)lane * 128u + ((uint32_t)(q ^ (lane & 7)) << 4);
+                    uint4 u = lds128(ad);
+                    float w0 = __uint_as_float(u.x), w1 = __uint_as_float(u.y), w2 = __uint_as_float(u.z),
+                          w3 = __uint_as_float(u.w);
+                    w0 = fmaf(-dsc.lr_eff, f[q * 4 + 0], fmaf(-dsc.wd_term, w0, w0));
+                    w1 = fmaf(-dsc.lr_eff, f[q * 4 + 1], fmaf(-dsc.wd_term, w1, w1));
+                    w2 = fmaf(-dsc.lr_eff, f[q * 4 + 2], fmaf(-dsc.wd_term, w2, w2));
+                    w3 = fmaf(-dsc.lr_eff, f[q * 4 + 3], fmaf(-dsc.wd_term, w3, w3));
+                    sts128(ad, make_uint4(__float_as_uint(w0), __float_as_uint(w1), __float_as_uint(w2),
+                                          __float_as_uint(w3)));
+                  }
+                } else {
+                  // block rows are tile columns: lane i reads element i of every row
+#pragma unroll
+                  for (int e = 0; e < 32; ++e) {
+                    const uint32_t ad = wb + (uint32_t)e * 128u + (uint32_t)lane * 4u;
+                    const float wv = __uint_as_float(lds32(ad));
+                    sts32(ad, __float_as_uint(fmaf(-dsc.lr_eff, f[e], fmaf(-dsc.wd_term, wv, wv))));
+                  }
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                  if (!dsc.transposed) tma_store_2d(dsc.wmap, wb, gjh, gi0);
+                  else tma_store_2d(dsc.wmap, wb, gi0, gjh);
+                  bulk_commit();
+                }
+                ++w_used;
+              }
+            } else if (gjh < p.N) {
               const MatDesc d = p.mats[mat];
               const bool full = (gi0 + 32 <= p.M) && (gjh + 32 <= p.N);
               if (full) {
@@ -620,6 +692,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
           }
         }
+        if (!alive) break;
         if (has_cin) ++cin_used;
         if (stores) {
           fence_async_smem();
@@ -692,6 +765,27 @@ bool encode_map(CUtensorMap* out, void* base, int64_t cols, int64_t rows, int64_
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
+
+}  // namespace
+
+bool tc_encode_w_map(void* out_host, void* base, int64_t rows, int64_t cols, int transposed) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn || (((uintptr_t)base) & 15) != 0 || (cols & 3) != 0) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap m;
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, transposed ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  static_assert(sizeof(CUtensorMap) == TC_MAP_BYTES, "TMA descriptor size");
+  memcpy(out_host, &m, sizeof m);
+  return true;
+}
+
+namespace {
 
 struct Maps5 {
   const CUtensorMap *a, *b, *c, *d, *t;
