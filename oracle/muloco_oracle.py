@@ -23,6 +23,8 @@ What each function follows:
   outer_nesterov       Eq. (3); Algorithm 1 lines 12-13
   quantize_blocks      Section 2 "Compressed Communication" (linear quantisation)
                        in the per-block absmax form of the benchmark configs
+  compressed_pseudogradient  Algorithm 2 (compression, error feedback) with the two
+                       quantisations of Section 2 "Collectives for compressed communication"
   fragments_due        Section 2 "Partitioned Communication in Streaming DiLoCo"
   MuLoCoOracle         Algorithm 1 (loop nest, initialisation line 2)
 
@@ -30,7 +32,8 @@ Pins (tests/test_oracle_*.py, all run without a GPU): SVD closed form of the
 Newton-Schulz map, exact rational iterates of the scalar quintic, rank-1 Muon
 step, K=1 equivalence with plain Muon, identical-gradient pseudogradient,
 Proposition 4.2's nuclear-norm identity, AdamW / outer-step closed forms,
-quantiser error bound / ties / idempotence, streaming coverage.
+quantiser error bound / ties / idempotence, streaming coverage, two-stage
+compression (K=1 collapse, error bound, error-feedback conservation).
 Parity unpinned: none of the functions above; the bf16 production mode of the
 GPU Newton-Schulz has no pin other than this oracle (tolerance 2e-2).
 """
@@ -191,6 +194,42 @@ def quantize_blocks(psi, bits: int, block: int = 128):
     return codes, scales, deq
 
 
+def compressed_pseudogradient(theta_g, thetas: Sequence[np.ndarray], bits: int, block: int = 128,
+                              ef: Optional[Sequence[np.ndarray]] = None, ef_beta: float = 1.0):
+    """Algorithm 2 with the two quantisations of Section 2 "Collectives for compressed
+    communication" (Appendix, "Assumptions around the collective used"), in float32:
+
+      per worker i:  Delta_i = theta - theta_i                       (parameter delta)
+                     with EF:  E_i <- beta E_i + Delta_i;  Delta~_i = C(E_i);  E_i <- E_i - Delta~_i
+                     else:     Delta~_i = C(Delta_i)                  (first quantisation, before
+                                                                       the all-to-all reduce-scatter)
+      Delta = (1/K) sum_i Delta~_i                                    (reduced in high precision)
+      Psi   = C(Delta)                                                (second quantisation, before
+                                                                       the all-gather)
+
+    C is quantize_blocks followed by dequantisation.  Every operation is a single float32
+    operation (no fused multiply-add), workers in ascending order, so that the integer
+    codes of both quantisations are reproducible bit for bit.  `ef` (float32 arrays, one
+    per worker) is updated in place.  Returns Psi (float32).
+    """
+    tg = np.asarray(theta_g, dtype=np.float32)
+    K = len(thetas)
+    acc = np.zeros_like(tg)
+    beta = np.float32(ef_beta)
+    for i, th in enumerate(thetas):
+        delta = (tg - np.asarray(th, dtype=np.float32)).astype(np.float32)
+        if ef is not None:
+            e = ((beta * ef[i]).astype(np.float32) + delta).astype(np.float32)
+            _, _, c = quantize_blocks(e, bits, block)
+            ef[i][...] = (e - c.reshape(e.shape)).astype(np.float32)
+        else:
+            _, _, c = quantize_blocks(delta, bits, block)
+        acc = (acc + c.reshape(tg.shape)).astype(np.float32)
+    mean = (acc * np.float32(1.0 / K)).astype(np.float32)
+    _, _, psi = quantize_blocks(mean, bits, block)
+    return psi.reshape(tg.shape)
+
+
 def pack_int4(codes):
     """Two 4-bit two's-complement codes per byte along a row, element 2j in the
     low nibble; a row with an odd number of elements pads the last high nibble
@@ -262,8 +301,12 @@ class OracleConfig:
     adam_bias_correction: bool = True
     outer_lr: float = 1.0
     outer_momentum: float = 0.0
-    quant_bits: int = 0           # 0 = none, 8, 4
-    quant_block: int = 128
+    quant_bits: int = 0           # 0 = none, 8, 4, 2
+    quant_block: int = 128        # 0 = one block per row (row-wise quantisation)
+    quant_stages: int = 1         # 1: quantise the averaged pseudogradient once (benchmark form);
+                                  # 2: per-worker quantisation, high-precision mean, second quantisation
+    error_feedback: bool = False  # Algorithm 2 (needs quant_stages = 2)
+    ef_beta: float = 1.0
 
     def f32(self) -> "OracleConfig":
         """The same configuration with every real hyper-parameter rounded to
@@ -271,7 +314,7 @@ class OracleConfig:
         r = lambda x: float(np.float32(x))
         d = dict(self.__dict__)
         for k in ("muon_lr", "muon_beta", "muon_wd", "ns_eps", "adam_lr", "adam_beta1",
-                  "adam_beta2", "adam_eps", "adam_wd", "outer_lr", "outer_momentum"):
+                  "adam_beta2", "adam_eps", "adam_wd", "outer_lr", "outer_momentum", "ef_beta"):
             d[k] = r(d[k])
         d["ns_coeffs"] = tuple(r(x) for x in self.ns_coeffs)
         return OracleConfig(**d)
@@ -298,6 +341,10 @@ class MuLoCoOracle:
         self.state1 = [[np.zeros_like(w) for w in self.theta_g] for _ in range(cfg.K)]
         self.state2 = [[np.zeros_like(w) if s.kind == "adamw" else None
                         for w, s in zip(self.theta_g, self.specs)] for _ in range(cfg.K)]
+        if cfg.error_feedback and (cfg.quant_stages != 2 or not cfg.quant_bits):
+            raise ValueError("error feedback needs the two-stage quantised sync")
+        # Algorithm 2 line 4: E_i <- 0
+        self.ef = [[np.zeros_like(w) for w in self.theta_g] for _ in range(cfg.K)] if cfg.error_feedback else None
         self.worker_step = [0] * cfg.K
         self.last_psi: Dict[int, np.ndarray] = {}
 
@@ -333,9 +380,13 @@ class MuLoCoOracle:
             if fragment >= 0 and s.fragment != fragment:
                 continue
             reps = [self.theta_k[k][i] for k in range(c.K)]
-            if c.quant_bits:
+            blk = c.quant_block if c.quant_block > 0 else s.cols
+            if c.quant_bits and c.quant_stages == 2:
+                efs = [self.ef[k][i] for k in range(c.K)] if self.ef is not None else None
+                psi = compressed_pseudogradient(self.theta_g[i], reps, c.quant_bits, blk, efs, c.ef_beta)
+            elif c.quant_bits:
                 psi32 = pseudogradient_f32(self.theta_g[i], reps)
-                _, _, psi = quantize_blocks(psi32, c.quant_bits, c.quant_block)
+                _, _, psi = quantize_blocks(psi32, c.quant_bits, blk)
             else:
                 psi = pseudogradient(self.theta_g[i], reps)
             self.last_psi[i] = np.array(psi)

@@ -333,3 +333,83 @@ def test_fragments_due_schedule():
     assert O.fragments_due(H, H, 1) == [0] and O.fragments_due(H - 1, H, 1) == []
     with pytest.raises(ValueError):
         O.fragments_due(1, 10, 4)
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 2: two-stage compression and error feedback
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("bits", [8, 4, 2])
+def test_two_stage_compression_collapses_for_one_worker(bits):
+    # K = 1: mean of one dequantised delta is that delta, and quantising a dequantised block
+    # again reproduces it (idempotence), so two stages equal one stage bit for bit
+    rng = np.random.default_rng(31 + bits)
+    tg = rng.standard_normal((5, 300)).astype(np.float32)
+    th = (tg - 0.01 * rng.standard_normal((5, 300))).astype(np.float32)
+    two = O.compressed_pseudogradient(tg, [th], bits, 128)
+    _, _, one = O.quantize_blocks((tg - th).astype(np.float32), bits, 128)
+    assert np.array_equal(two, one)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_two_stage_compression_error_bound(bits):
+    # each quantisation moves a value by at most half a step of its block: the result is within
+    # (mean of the workers' half steps) + (half step of the second stage) of the exact mean
+    rng = np.random.default_rng(7)
+    K, qmax = 4, (1 << (bits - 1)) - 1
+    tg = rng.standard_normal((3, 256)).astype(np.float32)
+    ths = [(tg - 0.02 * rng.standard_normal((3, 256))).astype(np.float32) for _ in range(K)]
+    psi = O.compressed_pseudogradient(tg, ths, bits, 128).astype(np.float64)
+    exact = np.mean([tg.astype(np.float64) - t for t in ths], axis=0)
+    for j in range(2):
+        sl = slice(128 * j, 128 * (j + 1))
+        half1 = np.mean([np.abs(tg[:, sl].astype(np.float64) - t[:, sl]).max(axis=1) / qmax / 2 for t in ths], axis=0)
+        half2 = (np.abs(exact[:, sl]).max(axis=1) + half1) / qmax / 2
+        bound = (half1 + half2)[:, None] * (1 + 1e-5) + 1e-7
+        assert np.all(np.abs(psi[:, sl] - exact[:, sl]) <= bound)
+
+
+def test_error_feedback_conserves_what_was_not_sent():
+    # beta = 1: after every sync  E_i + (sum of everything sent so far) = sum of the deltas so far,
+    # up to one float32 rounding per operation; and |E_i| is at most half a quantisation step
+    rng = np.random.default_rng(11)
+    K, bits = 2, 4
+    tg = np.zeros((2, 128), dtype=np.float32)
+    ef = [np.zeros_like(tg) for _ in range(K)]
+    sent = [np.zeros(tg.shape) for _ in range(K)]
+    total = [np.zeros(tg.shape) for _ in range(K)]
+    for rnd in range(6):
+        ths = [(-(0.1 * rng.standard_normal(tg.shape))).astype(np.float32) for _ in range(K)]   # delta_i = -theta_i
+        before = [e.copy() for e in ef]
+        O.compressed_pseudogradient(tg, ths, bits, 128, ef, 1.0)
+        for i in range(K):
+            e_in = (before[i] + (tg - ths[i])).astype(np.float32)
+            c = e_in.astype(np.float64) - ef[i]                     # what worker i sent this round
+            _, sc, deq = O.quantize_blocks(e_in, bits, 128)
+            assert np.allclose(c, deq, rtol=0, atol=1e-6 * np.abs(e_in).max())
+            assert np.all(np.abs(ef[i]) <= sc[:, :1] / 2 * (1 + 1e-5) + 1e-7)
+            sent[i] += c
+            total[i] += (tg - ths[i]).astype(np.float64)
+            assert np.allclose(sent[i] + ef[i], total[i], rtol=0, atol=1e-5)
+
+
+def test_error_feedback_changes_nothing_when_nothing_is_lost():
+    # values that the quantiser represents exactly (multiples of the step, absmax = 7 steps)
+    # leave E = 0, and the sync equals the uncompressed mean
+    steps = np.array([[7, -3, 0, 1, 5, -7, 2, 4]], dtype=np.float32)
+    tg = np.zeros((1, 8), dtype=np.float32)
+    ths = [-(0.25 * steps), -(0.5 * steps[:, ::-1].copy())]
+    ef = [np.zeros_like(tg) for _ in range(2)]
+    psi = O.compressed_pseudogradient(tg, [t.astype(np.float32) for t in ths], 4, 8, ef, 0.9)
+    assert all(np.all(e == 0) for e in ef)
+    mean = (0.25 * steps + 0.5 * steps[:, ::-1]) / 2
+    _, _, want = O.quantize_blocks(mean.astype(np.float32), 4, 8)
+    assert np.array_equal(psi, want)
+
+
+def test_row_wise_quantisation_is_one_block_per_row():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((4, 300)).astype(np.float32)
+    codes, scales, deq = O.quantize_blocks(x, 8, 300)
+    assert scales.shape == (4, 1)
+    assert np.array_equal(scales[:, 0], (np.abs(x).max(axis=1) / np.float32(127)).astype(np.float32))
+    assert np.all(np.abs(codes).max(axis=1) == 127)
