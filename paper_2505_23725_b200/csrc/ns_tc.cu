@@ -48,13 +48,17 @@ constexpr int BM = 128;          // rows per CTA (one CTA's share of UMMA M)
 constexpr int BK = 64;           // k slab per stage (64 bf16 = one 128-byte swizzle row)
 constexpr int UMMA_K = 16;
 constexpr int TC_THREADS = 192;
-constexpr int STAGES = 4;
+// Pipeline depth is a template parameter: products that need all six staging blocks per epilogue
+// warp (POLY: addend + direct + mirrored; FINAL: addend + parameter ring) run 4 stages, those that
+// need four (GRAM: direct + mirrored; APPLY: addend + direct) run 5 in the same shared memory.
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;        // 16 KB: 128 rows x 64 k
 constexpr uint32_t B_STAGE_BYTES = 128 * BK * 2;       // 16 KB: this CTA's 128 columns of the right operand
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr uint32_t EPI_BLOCK_BYTES = 32 * 64 * 2;      // one 32 x 64 bf16 block
-constexpr uint32_t EPI_WARP_BYTES = 6 * EPI_BLOCK_BYTES;   // addend x2, direct x2, mirrored x2
-constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_WARP_BYTES + 1024;   // + alignment slack
+__host__ __device__ constexpr uint32_t epi_warp_bytes(int nstg) { return (nstg == 5 ? 4u : 6u) * EPI_BLOCK_BYTES; }
+__host__ __device__ constexpr uint32_t smem_bytes(int nstg) {
+  return (uint32_t)nstg * STAGE_BYTES + 4u * epi_warp_bytes(nstg) + 1024u;   // + alignment slack
+}
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 struct TcParams {
@@ -278,7 +282,7 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
 // tmC     : addend loads, 64 x 32 boxes (POLY: A, APPLY/FINAL: X)
 // tmD     : result stores, 64 x 32 boxes, 128-byte swizzle
 // tmT     : transposed result stores, 32 x 64 boxes, no swizzle (symmetric products)
-template <int CG, bool B_MN>
+template <int CG, bool B_MN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
@@ -440,11 +444,12 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // -------------------------------- epilogue --------------------------------
     const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter+32)
     const int ew = warp - 2;               // staging slot of this warp
-    const uint32_t epi = smem_base + STAGES * STAGE_BYTES + (uint32_t)ew * EPI_WARP_BYTES;
+    const uint32_t epi = smem_base + STAGES * STAGE_BYTES + (uint32_t)ew * epi_warp_bytes(STAGES);
     // staging blocks of this warp: addend 0/1, direct 0/1, mirrored 0/1
     auto cin_buf = [&](uint32_t b) { return epi + b * EPI_BLOCK_BYTES; };
-    auto out_buf = [&](uint32_t b) { return epi + (2u + b) * EPI_BLOCK_BYTES; };
-    auto mir_buf = [&](uint32_t b) { return epi + (4u + b) * EPI_BLOCK_BYTES; };
+    const uint32_t o_first = (p.kind == GEMM_GRAM) ? 0u : 2u;     // the addend blocks come first when there are any
+    auto out_buf = [&](uint32_t b) { return epi + (o_first + b) * EPI_BLOCK_BYTES; };
+    auto mir_buf = [&](uint32_t b) { return epi + (o_first + 2u + b) * EPI_BLOCK_BYTES; };
     const uint32_t cin_bar0 = smem_u32(&bar_cin[ew][0]);
     auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
     const bool has_cin = (p.kind != GEMM_GRAM);
@@ -792,13 +797,13 @@ struct Maps5 {
 };
 
 // Number of tile workers (CTAs for CG = 1, CTA pairs for CG = 2) that can be resident at once.
-template <int CG, bool B_MN>
+template <int CG, bool B_MN, int NSTG>
 int resident_units(int n_sms, cudaError_t* err) {
   static int cached = 0;
   *err = cudaSuccess;
   if (cached) return cached;
-  cudaError_t e = cudaFuncSetAttribute(ns_tc_kernel<CG, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(ns_tc_kernel<CG, B_MN, NSTG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem_bytes(NSTG));
   if (e != cudaSuccess) { *err = e; return 0; }
   if (CG == 1) {
     cached = n_sms;
@@ -808,23 +813,23 @@ int resident_units(int n_sms, cudaError_t* err) {
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)(n_sms / 2 * 2));
   cfg.blockDim = dim3(TC_THREADS);
-  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.dynamicSmemBytes = smem_bytes(NSTG);
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, ns_tc_kernel<CG, B_MN>, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&n, ns_tc_kernel<CG, B_MN, NSTG>, &cfg);
   if (e != cudaSuccess) { *err = e; return 0; }
   if (n < 1) { *err = cudaErrorLaunchOutOfResources; return 0; }
   cached = n;
   return cached;
 }
 
-template <int CG, bool B_MN>
+template <int CG, bool B_MN, int NSTG>
 cudaError_t launch_one(cudaStream_t st, const Maps5& m, const TcParams& p, int n_sms) {
   cudaError_t e;
-  const int units = resident_units<CG, B_MN>(n_sms, &e);
+  const int units = resident_units<CG, B_MN, NSTG>(n_sms, &e);
   if (e != cudaSuccess) return e;
   const int total = p.n_mats * p.n_tiles_per_mat;
   const int workers = total < units ? total : units;
@@ -832,13 +837,13 @@ cudaError_t launch_one(cudaStream_t st, const Maps5& m, const TcParams& p, int n
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)(workers * CG));
   cfg.blockDim = dim3(TC_THREADS);
-  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.dynamicSmemBytes = smem_bytes(NSTG);
   cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, ns_tc_kernel<CG, B_MN>, *m.a, *m.b, *m.c, *m.d, *m.t, p);
+  return cudaLaunchKernelEx(&cfg, ns_tc_kernel<CG, B_MN, NSTG>, *m.a, *m.b, *m.c, *m.d, *m.t, p);
 }
 
 }  // namespace
@@ -935,17 +940,19 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int kind, int n_mats, in
   if (kind == GEMM_GRAM) {
     p.N = (int)pl->s; p.Kd = (int)pl->l; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
     m = Maps5{&pl->x_k[xin], &pl->x_k[xin], &pl->a_io, &pl->a_io, &pl->a_tr};
-    return pl->cg == 2 ? launch_one<2, false>(st, m, p, pl->n_sms) : launch_one<1, false>(st, m, p, pl->n_sms);
+    return pl->cg == 2 ? launch_one<2, false, 5>(st, m, p, pl->n_sms) : launch_one<1, false, 5>(st, m, p, pl->n_sms);
   }
   if (kind == GEMM_POLY) {
     p.N = (int)pl->s; p.Kd = (int)pl->s; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
     m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, &pl->b_tr};
-    return pl->cg == 2 ? launch_one<2, false>(st, m, p, pl->n_sms) : launch_one<1, false>(st, m, p, pl->n_sms);
+    return pl->cg == 2 ? launch_one<2, false, 4>(st, m, p, pl->n_sms) : launch_one<1, false, 4>(st, m, p, pl->n_sms);
   }
   p.N = (int)pl->l; p.Kd = (int)pl->s; p.tiles = pl->tiles_full; p.n_tiles_per_mat = pl->n_tiles_full;
   // FINAL stores nothing through tmD; the map still has to be a valid one
   m = Maps5{&pl->b_k, &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin], &pl->x_io[1 - xin]};
-  return pl->cg == 2 ? launch_one<2, true>(st, m, p, pl->n_sms) : launch_one<1, true>(st, m, p, pl->n_sms);
+  if (kind == GEMM_APPLY)
+    return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
+  return pl->cg == 2 ? launch_one<2, true, 4>(st, m, p, pl->n_sms) : launch_one<1, true, 4>(st, m, p, pl->n_sms);
 }
 
 }  // namespace muloco
