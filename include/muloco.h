@@ -55,7 +55,7 @@ typedef enum {
 
 typedef enum { MULOCO_MUON = 0, MULOCO_ADAMW = 1 } muloco_kind;
 typedef enum { MULOCO_NS_BF16 = 0, MULOCO_NS_FP32 = 1 } muloco_ns_mode;
-typedef enum { MULOCO_Q_NONE = 0, MULOCO_Q_INT4 = 4, MULOCO_Q_INT8 = 8 } muloco_quant;
+typedef enum { MULOCO_Q_NONE = 0, MULOCO_Q_INT2 = 2, MULOCO_Q_INT4 = 4, MULOCO_Q_INT8 = 8 } muloco_quant;
 typedef enum { MULOCO_F32 = 0, MULOCO_BF16 = 1 } muloco_dtype;
 
 /* One parameter tensor of the model. */
@@ -87,8 +87,16 @@ typedef struct {
   int32_t quant;       /* muloco_quant: quantise -> dequantise the pseudogradient       */
   int32_t quant_block; /* elements per absmax block along a row (128)                   */
   int32_t grad_dtype;  /* muloco_dtype of the gradients given to muloco_inner_step      */
-  int32_t reserved;
+  int32_t quant_stages; /* 0 or 1: quantise the averaged pseudogradient once (benchmark form);
+                           2: Algorithm 2 with the two quantisations of Section 2
+                           ("Collectives for compressed communication"): every worker's delta
+                           is quantised, the mean is taken in float32, the mean is quantised
+                           again                                                            */
   uint64_t workspace_bytes; /* Newton-Schulz workspace budget; 0 lets the library pick  */
+  int32_t error_feedback; /* 1: Algorithm 2's error feedback, E_i <- beta E_i + Delta_i,
+                             send C(E_i), E_i <- E_i - C(E_i); needs quant_stages == 2 and
+                             the ef_k buffers                                              */
+  float ef_beta;       /* beta of the error-feedback accumulator                          */
 } muloco_config;
 
 /* State buffers.  Every field is a HOST array of DEVICE pointers.
@@ -99,6 +107,8 @@ typedef struct {
   float* const* outer_u;  /* [n]     outer momentum u                                   */
   float* const* state1_k; /* [K][n]  Muon momentum m, or Adam first moment              */
   float* const* state2_k; /* [K][n]  Adam second moment (ignored for Muon tensors)      */
+  float* const* ef_k;     /* [K][n]  error-feedback accumulators E_i (Algorithm 2); the table
+                             may be NULL unless cfg.error_feedback is set                */
 } muloco_buffers;
 
 /* Algorithm 1, line 2.  Validates the arguments, records the tensor table,
@@ -138,7 +148,11 @@ MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* ctx, int32_t worker,
  * (0..J-1), or all tensors when fragment == -1, in one pass over memory:
  *     Psi = (1/K) sum_k (theta_g - theta_k)   (fp32, k ascending, then * 1/K)
  *     optional: Psi <- dequantise(quantise(Psi)) per block of quant_block elements
- *               along a row (absmax scale, round to nearest even, int8 or int4)
+ *               along a row (absmax scale, round to nearest even, int8, int4 or int2)
+ *     with quant_stages == 2 (Algorithm 2): every worker's delta theta_g - theta_k (or, with
+ *               error feedback, E_k <- ef_beta E_k + delta) is quantised -> dequantised first
+ *               (and E_k <- E_k - what was sent), the mean of those is taken in fp32 (k
+ *               ascending, then * 1/K) and quantised -> dequantised again
  *     u <- mu u + eta_out Psi;   theta_g <- theta_g - mu u - eta_out Psi
  *     theta_k <- theta_g for every worker.
  * Inner optimizer state is kept.  Syncing a fragment that is not due is allowed;
@@ -206,7 +220,7 @@ MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, float* O, i
  * rows x cols float32 matrix; writes, where non-NULL, one int8 code per element
  * to `codes` (int4 codes are -7..7, unpacked), one float32 scale per block to
  * `scales` ([rows][ceil(cols/block)]) and the dequantised values to `dequant`.
- * bits is 8 or 4. */
+ * bits is 8, 4 or 2. */
 MULOCO_API muloco_status muloco_quantize(muloco_ctx* ctx, const float* psi, int64_t rows, int64_t cols,
                               int32_t bits, int8_t* codes, float* scales, float* dequant);
 

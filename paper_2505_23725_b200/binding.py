@@ -51,13 +51,14 @@ class Config(C.Structure):
                 ("adam_eps", C.c_float), ("adam_wd", C.c_float), ("adam_bias_correction", C.c_int32),
                 ("outer_lr", C.c_float), ("outer_momentum", C.c_float),
                 ("quant", C.c_int32), ("quant_block", C.c_int32), ("grad_dtype", C.c_int32),
-                ("reserved", C.c_int32), ("workspace_bytes", C.c_uint64)]
+                ("quant_stages", C.c_int32), ("workspace_bytes", C.c_uint64),
+                ("error_feedback", C.c_int32), ("ef_beta", C.c_float)]
 
 
 class Buffers(C.Structure):
     _fields_ = [("theta_k", C.POINTER(C.c_void_p)), ("theta_g", C.POINTER(C.c_void_p)),
                 ("outer_u", C.POINTER(C.c_void_p)), ("state1_k", C.POINTER(C.c_void_p)),
-                ("state2_k", C.POINTER(C.c_void_p))]
+                ("state2_k", C.POINTER(C.c_void_p)), ("ef_k", C.POINTER(C.c_void_p))]
 
 
 class MulocoError(RuntimeError):
@@ -146,6 +147,9 @@ def make_config(w: _cfg.Workload, workspace_bytes: int = 0, ns_mode: Optional[st
     c.outer_lr, c.outer_momentum = w.outer_lr, w.outer_momentum
     c.quant = w.quant_bits
     c.quant_block = w.quant_block
+    c.quant_stages = w.quant_stages
+    c.error_feedback = int(w.error_feedback)
+    c.ef_beta = w.ef_beta
     c.grad_dtype = BF16 if w.grad_dtype == "bf16" else F32
     c.workspace_bytes = workspace_bytes
     for k, v in over.items():
@@ -198,6 +202,9 @@ class MuLoCo:
         self.flat_s1 = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)]
         self.flat_s2 = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)] \
             if any(t.kind == _cfg.ADAMW for t in workload.tensors) else [None] * self.K
+        self.flat_ef = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)] \
+            if workload.error_feedback else None
+        self.ef = [self._views(b) for b in self.flat_ef] if self.flat_ef else None
         self.theta_g = self._views(self.flat_theta_g)
         self.outer_u = self._views(self.flat_u)
         self.theta_k = [self._views(b) for b in self.flat_theta_k]
@@ -239,6 +246,9 @@ class MuLoCo:
         ]
         bufs.theta_k, bufs.theta_g, bufs.outer_u, bufs.state1_k, bufs.state2_k = [
             C.cast(t, C.POINTER(C.c_void_p)) for t in self._tables]
+        if self.ef is not None:
+            self._tables.append(_ptr_table([self.ef[k][i].data_ptr() for k in range(self.K) for i in range(self.n)]))
+            bufs.ef_k = C.cast(self._tables[-1], C.POINTER(C.c_void_p))
         self.stream = stream if stream is not None else torch.cuda.current_stream(dev)
         self.ctx = C.c_void_p()
         st = self.lib.muloco_create(C.byref(self.cfg), descs, self.n, C.byref(bufs),

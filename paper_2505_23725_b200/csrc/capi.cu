@@ -26,7 +26,7 @@ struct TensorInfo {
   float wd_mult, lr_mult;
   float* theta_g;
   float* u;
-  std::vector<float*> theta_k, s1, s2;
+  std::vector<float*> theta_k, s1, s2, ef;
   int64_t numel() const { return rows * cols; }
 };
 
@@ -99,6 +99,7 @@ struct muloco_ctx {
 
   std::vector<FragTable> frags;   // J entries + one for "all"
   float** d_replicas = nullptr;   // [n][K]
+  float** d_ef = nullptr;         // [n][K] error-feedback accumulators (Algorithm 2), or NULL
 
   // per-call tables
   MatDesc* d_mats = nullptr;
@@ -187,8 +188,15 @@ muloco_status validate_config(const muloco_config* cfg) {
   if (cfg->ns_steps < 1 || cfg->ns_steps > 64) return fail(c, MULOCO_EINVAL, "ns_steps must be in 1..64");
   if (cfg->ns_mode != MULOCO_NS_BF16 && cfg->ns_mode != MULOCO_NS_FP32)
     return fail(c, MULOCO_EINVAL, "unknown ns_mode %d", cfg->ns_mode);
-  if (cfg->quant != MULOCO_Q_NONE && cfg->quant != MULOCO_Q_INT4 && cfg->quant != MULOCO_Q_INT8)
-    return fail(c, MULOCO_EINVAL, "quant must be 0, 4 or 8");
+  if (cfg->quant != MULOCO_Q_NONE && cfg->quant != MULOCO_Q_INT2 && cfg->quant != MULOCO_Q_INT4 &&
+      cfg->quant != MULOCO_Q_INT8)
+    return fail(c, MULOCO_EINVAL, "quant must be 0, 2, 4 or 8");
+  if (cfg->quant_stages < 0 || cfg->quant_stages > 2)
+    return fail(c, MULOCO_EINVAL, "quant_stages must be 0, 1 or 2");
+  if (cfg->error_feedback != 0 && (cfg->quant_stages != 2 || cfg->quant == MULOCO_Q_NONE))
+    return fail(c, MULOCO_EINVAL, "error_feedback needs quant_stages == 2 and a quantiser");
+  if (cfg->error_feedback != 0 && !(cfg->ef_beta >= 0.f && cfg->ef_beta <= 1.f))
+    return fail(c, MULOCO_EINVAL, "ef_beta must be in [0, 1]");
   if (!valid_block(cfg->quant_block)) return fail(c, MULOCO_EINVAL, "quant_block must be 32, 64 or 128");
   if (cfg->grad_dtype != MULOCO_F32 && cfg->grad_dtype != MULOCO_BF16)
     return fail(c, MULOCO_EINVAL, "unknown grad_dtype %d", cfg->grad_dtype);
@@ -279,6 +287,12 @@ muloco_status build_sync_tables(muloco_ctx* c) {
   if (n > 0) {
     CK(cudaMalloc(&c->d_replicas, reps.size() * sizeof(float*)));
     CK(cudaMemcpy(c->d_replicas, reps.data(), reps.size() * sizeof(float*), cudaMemcpyHostToDevice));
+    if (c->cfg.error_feedback != 0) {
+      for (int i = 0; i < n; ++i)
+        for (int k = 0; k < K; ++k) reps[(size_t)i * K + k] = c->T[i].ef[k];
+      CK(cudaMalloc(&c->d_ef, reps.size() * sizeof(float*)));
+      CK(cudaMemcpy(c->d_ef, reps.data(), reps.size() * sizeof(float*), cudaMemcpyHostToDevice));
+    }
   }
   c->frags.resize(c->cfg.J + 1);
   for (int f = 0; f <= c->cfg.J; ++f) {
@@ -344,6 +358,8 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
                         !bufs->state1_k || !bufs->state2_k))
     return fail(c, MULOCO_EINVAL, "tensor table or buffer table is NULL");
   const int K = cfg->K;
+  if (n_tensors > 0 && cfg->error_feedback != 0 && !bufs->ef_k)
+    return fail(c, MULOCO_EINVAL, "error_feedback is set but the ef_k table is NULL");
   for (int i = 0; i < n_tensors; ++i) {
     const muloco_tensor_desc& d = tensors[i];
     if (d.rows < 1 || d.cols < 1) return fail(c, MULOCO_ESHAPE, "tensor %d has an empty shape", i);
@@ -359,6 +375,8 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
       if (!bufs->theta_k[e] || !bufs->state1_k[e]) return fail(c, MULOCO_EINVAL, "tensor %d worker %d: NULL buffer", i, k);
       if (d.kind == MULOCO_ADAMW && !bufs->state2_k[e])
         return fail(c, MULOCO_EINVAL, "tensor %d worker %d: NULL second-moment buffer", i, k);
+      if (cfg->error_feedback != 0 && !bufs->ef_k[e])
+        return fail(c, MULOCO_EINVAL, "tensor %d worker %d: NULL error-feedback buffer", i, k);
     }
   }
   int ndev = 0;
@@ -403,6 +421,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
       t.theta_k.push_back(bufs->theta_k[e]);
       t.s1.push_back(bufs->state1_k[e]);
       t.s2.push_back(d.kind == MULOCO_ADAMW ? bufs->state2_k[e] : nullptr);
+      t.ef.push_back(cfg->error_feedback != 0 ? bufs->ef_k[e] : nullptr);
     }
     (d.kind == MULOCO_MUON ? c->muon_ids : c->adam_ids).push_back(i);
   }
@@ -482,6 +501,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
     for (int k = 0; k < K; ++k) {
       CKC(cudaMemsetAsync(t.s1[k], 0, bytes, c->st));
       if (t.s2[k]) CKC(cudaMemsetAsync(t.s2[k], 0, bytes, c->st));
+      if (t.ef[k]) CKC(cudaMemsetAsync(t.ef[k], 0, bytes, c->st));     // Algorithm 2: E_i <- 0
       CKC(cudaMemcpyAsync(t.theta_k[k], t.theta_g, bytes, cudaMemcpyDeviceToDevice, c->st));
     }
   }
@@ -500,6 +520,7 @@ MULOCO_API void muloco_destroy(muloco_ctx* c) {
   if (c->sa_d_mats) cudaFree(c->sa_d_mats);
   if (c->d_status) cudaFree(c->d_status);
   if (c->d_replicas) cudaFree(c->d_replicas);
+  if (c->d_ef) cudaFree(c->d_ef);
   if (c->d_mats) cudaFree(c->d_mats);
   if (c->d_adam) cudaFree(c->d_adam);
   if (c->d_wmaps) cudaFree(c->d_wmaps);
@@ -652,7 +673,7 @@ MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* c, int32_t fragment) {
   PhaseTimer t(c, MULOCO_PH_SYNC);
   const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
   launch_outer_sync(c->st, ft.d_segs, ft.n_segs, c->d_replicas, f.K, ft.n_units, blk, f.quant, f.outer_lr,
-                    f.outer_momentum, c->d_status, c->n_sms);
+                    f.outer_momentum, c->d_status, c->n_sms, f.quant_stages == 2 ? 2 : 1, c->d_ef, f.ef_beta);
   c->launches += 1;
   CK(cudaGetLastError());
   return MULOCO_OK;
@@ -755,7 +776,7 @@ MULOCO_API muloco_status muloco_quantize(muloco_ctx* c, const float* psi, int64_
                               int8_t* codes, float* scales, float* dequant) {
   if (!c) return MULOCO_EINVAL;
   if (!psi) return fail(c, MULOCO_EINVAL, "psi is NULL");
-  if (bits != 8 && bits != 4) return fail(c, MULOCO_EINVAL, "bits must be 8 or 4");
+  if (bits != 8 && bits != 4 && bits != 2) return fail(c, MULOCO_EINVAL, "bits must be 8, 4 or 2");
   if (rows < 0 || cols < 0) return fail(c, MULOCO_ESHAPE, "negative shape");
   if (rows == 0 || cols == 0) return MULOCO_OK;
   launch_quantize(c->st, psi, rows, cols, c->cfg.quant_block, bits, codes, scales, dequant, c->d_status);

@@ -96,9 +96,12 @@ struct SyncSeg {
   int64_t unit_begin;   // first block-unit of this segment
   int64_t rep_index;    // index of this tensor's first replica pointer in the replica table
 };
+// ef: table of error-feedback accumulators laid out like `replicas` (NULL: no error feedback);
+// stages 2 selects the per-worker quantisation of Algorithm 2.
 void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
                        int K, int64_t n_units, int block, int quant_bits, float outer_lr,
-                       float mu, int* status, int n_sms);
+                       float mu, int* status, int n_sms, int stages = 1, float* const* ef = nullptr,
+                       float ef_beta = 1.0f);
 void launch_pseudogradient(cudaStream_t st, const float* theta_g, float* const* replicas, int K,
                            int64_t n, float* psi_out);
 void launch_quantize(cudaStream_t st, const float* psi, int64_t rows, int64_t cols, int block,

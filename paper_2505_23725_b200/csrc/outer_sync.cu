@@ -43,7 +43,7 @@ __device__ __forceinline__ float warp_max(float v) {
 template <int QB>
 __device__ __forceinline__ void quant_dequant4(float (&x)[4], int nvalid, int (&q)[4], float& scale,
                                                bool& bad) {
-  constexpr float qmax = (QB == 8) ? 127.0f : 7.0f;
+  constexpr float qmax = (QB == 8) ? 127.0f : (QB == 4 ? 7.0f : 1.0f);
   float lmax = 0.0f;
 #pragma unroll
   for (int e = 0; e < 4; ++e)
@@ -193,6 +193,112 @@ outer_sync_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __
   if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
 }
 
+// Algorithm 2 with two quantisations (Section 2, "Collectives for compressed communication"):
+// every worker's delta (or error-feedback accumulator) is quantised -> dequantised per block,
+// the mean of those is taken in fp32 (k ascending, then * 1/K) and quantised again.  Workers are
+// read four at a time.  Same unit/CTA mapping as outer_sync_kernel; with error feedback the
+// accumulators add one fp32 read and one write per worker and parameter.
+template <int QB, bool EF>
+__global__ void __launch_bounds__(SYNC_THREADS)
+outer_sync2_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps,
+                   float* const* __restrict__ efs, int K, int64_t n_units, int64_t units_per_cta, int block,
+                   float eta, float mu, float inv_k, float ef_beta, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t cta_begin = (int64_t)blockIdx.x * units_per_cta;
+  int64_t cta_end = cta_begin + units_per_cta;
+  if (cta_end > n_units) cta_end = n_units;
+  bool bad = false;
+  int64_t unit = cta_begin + warp;
+  if (unit < cta_end) {
+    int seg = find_seg(segs, n_segs, unit);
+    SyncSeg s = segs[seg];
+    int64_t seg_end = (seg + 1 < n_segs) ? segs[seg + 1].unit_begin : n_units;
+    for (; unit < cta_end; unit += SYNC_WARPS) {
+      while (unit >= seg_end) {
+        ++seg;
+        s = segs[seg];
+        seg_end = (seg + 1 < n_segs) ? segs[seg + 1].unit_begin : n_units;
+      }
+      const int64_t ul = unit - s.unit_begin;
+      const int64_t row = ul / s.nblk;
+      const int64_t blk = ul - row * s.nblk;
+      const int64_t col0 = blk * block + lane * 4;
+      int64_t blk_end = (blk + 1) * block;
+      if (blk_end > s.cols) blk_end = s.cols;
+      int nvalid = (int)(blk_end - col0);
+      nvalid = nvalid < 0 ? 0 : (nvalid > 4 ? 4 : nvalid);
+      const int64_t off = row * s.cols + col0;
+      float* const* rp = reps + s.rep_index;
+      float* const* ep = EF ? efs + s.rep_index : nullptr;
+      bool vec = ((s.cols & 3) == 0) && ((((uintptr_t)s.theta_g | (uintptr_t)s.u) & 15) == 0) && nvalid == 4;
+      for (int k = 0; k < K; ++k) {
+        vec = vec && ((((uintptr_t)rp[k]) & 15) == 0);
+        if (EF) vec = vec && ((((uintptr_t)ep[k]) & 15) == 0);
+      }
+      float tg[4] = {0.f, 0.f, 0.f, 0.f}, uu[4] = {0.f, 0.f, 0.f, 0.f}, acc[4] = {0.f, 0.f, 0.f, 0.f};
+      if (nvalid > 0) {
+        load4(s.theta_g + off, vec, nvalid, tg);
+        load4(s.u + off, vec, nvalid, uu);
+      }
+      for (int k0 = 0; k0 < K; k0 += 4) {
+        float r[4][4], e[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { r[j][q] = 0.f; e[j][q] = 0.f; }
+          if (k0 + j < K && nvalid > 0) {
+            load4(rp[k0 + j] + off, vec, nvalid, r[j]);
+            if (EF) load4(ep[k0 + j] + off, vec, nvalid, e[j]);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (k0 + j < K) {            // uniform over the warp: the block reduction below needs every lane
+            float x[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float d = __fsub_rn(tg[q], r[j][q]);
+              x[q] = EF ? __fadd_rn(__fmul_rn(ef_beta, e[j][q]), d) : d;
+            }
+            float sent[4] = {x[0], x[1], x[2], x[3]};
+            int qq[4]; float sc;
+            quant_dequant4<QB>(sent, nvalid, qq, sc, bad);
+            if (EF && nvalid > 0) {
+              float en[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) en[q] = __fsub_rn(x[q], sent[q]);
+              store4(ep[k0 + j] + off, vec, nvalid, en);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], sent[q]);
+          }
+        }
+      }
+      float psi[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) psi[q] = __fmul_rn(acc[q], inv_k);
+      {
+        int qq[4]; float sc;
+        quant_dequant4<QB>(psi, nvalid, qq, sc, bad);
+      }
+      if (nvalid > 0) {
+        float un[4], tn[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float epq = eta * psi[q];
+          un[q] = fmaf(mu, uu[q], epq);
+          tn[q] = tg[q] - fmaf(mu, un[q], epq);
+        }
+        store4(s.u + off, vec, nvalid, un);
+        store4(s.theta_g + off, vec, nvalid, tn);
+        for (int k = 0; k < K; ++k) store4(rp[k] + off, vec, nvalid, tn);
+      }
+    }
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
+}
+
 __global__ void pseudograd_kernel(const float* __restrict__ tg, float* const* __restrict__ reps, int K,
                                   int64_t n, float inv_k, float* __restrict__ out) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -269,17 +375,35 @@ void launch_sync_q(cudaStream_t st, dim3 grid, const SyncSeg* segs, int n_segs, 
 
 void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
                        int K, int64_t n_units, int block, int quant_bits, float outer_lr, float mu,
-                       int* status, int n_sms) {
+                       int* status, int n_sms, int stages, float* const* ef, float ef_beta) {
   (void)n_sms;
   if (n_units <= 0) return;
   const int64_t upc = (int64_t)SYNC_WARPS * SYNC_UNITS_PER_WARP;
   const int64_t ctas = (n_units + upc - 1) / upc;
   const float inv_k = 1.0f / (float)K;
   dim3 grid((unsigned)ctas);
+  if (stages == 2 && quant_bits != 0) {
+#define MULOCO_SYNC2_CASE(QB)                                                                        \
+  do {                                                                                             \
+    if (ef)                                                                                        \
+      outer_sync2_kernel<QB, true><<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, replicas, ef, K, n_units, upc, \
+                                                                  block, outer_lr, mu, inv_k, ef_beta, status); \
+    else                                                                                           \
+      outer_sync2_kernel<QB, false><<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, replicas, ef, K, n_units, upc, \
+                                                                   block, outer_lr, mu, inv_k, ef_beta, status); \
+  } while (0)
+    if (quant_bits == 8) MULOCO_SYNC2_CASE(8);
+    else if (quant_bits == 4) MULOCO_SYNC2_CASE(4);
+    else MULOCO_SYNC2_CASE(2);
+#undef MULOCO_SYNC2_CASE
+    return;
+  }
   if (quant_bits == 8)
     launch_sync_q<8>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
   else if (quant_bits == 4)
     launch_sync_q<4>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+  else if (quant_bits == 2)
+    launch_sync_q<2>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
   else
     launch_sync_q<0>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
 }
@@ -299,6 +423,8 @@ void launch_quantize(cudaStream_t st, const float* psi, int64_t rows, int64_t co
   int blocks = (int)((n_units + 7) / 8 < 4096 ? (n_units + 7) / 8 : 4096);
   if (bits == 8)
     quantize_kernel<8><<<blocks, 256, 0, st>>>(psi, rows, cols, block, nblk, codes, scales, dequant, status);
+  else if (bits == 2)
+    quantize_kernel<2><<<blocks, 256, 0, st>>>(psi, rows, cols, block, nblk, codes, scales, dequant, status);
   else
     quantize_kernel<4><<<blocks, 256, 0, st>>>(psi, rows, cols, block, nblk, codes, scales, dequant, status);
 }

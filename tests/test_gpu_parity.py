@@ -370,3 +370,76 @@ def test_argument_errors_are_reported_on_the_host():
     with pytest.raises(binding.MulocoError):
         gpu.inner_step(7, [gpu.theta_g[i] for i in range(gpu.n)])
     gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 2: two quantisations per sync, optional error feedback, 2-bit codes
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("K", [1, 2, 4, 5, 16])
+@pytest.mark.parametrize("bits,ef", [(8, False), (4, False), (2, False), (4, True), (8, True), (2, True)])
+def test_two_stage_quantised_sync_vs_oracle(K, bits, ef):
+    import dataclasses
+    import torch
+    w = dataclasses.replace(_sync_workload(K, bits, SYNC_SHAPES), quant_stages=2, error_feedback=ef, ef_beta=0.9)
+    rng = np.random.default_rng(500 + 10 * K + bits + ef)
+    init = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) * 0.02 for t in w.tensors]
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init, quant_stages=2, error_feedback=ef, ef_beta=0.9)
+    for rnd in range(3):                                   # three syncs: accumulators and momentum carry over
+        for k in range(K):
+            for i, t in enumerate(w.tensors):
+                drift = (rng.standard_normal((t.rows, t.cols)) * 10.0 ** rng.uniform(-4, -1)).astype(np.float32)
+                orc.theta_k[k][i][...] = orc.theta_g[i] + drift
+                gpu.theta_k[k][i].copy_(torch.from_numpy(orc.theta_k[k][i]).cuda())
+        gpu.outer_sync(-1)
+        orc.outer_sync(-1)
+        gpu.sync_status()
+        for i in range(gpu.n):
+            if ef:
+                for k in range(K):                         # accumulators: exact float32 arithmetic on both sides
+                    assert np.array_equal(_np(gpu.ef[k][i]), orc.ef[k][i]), f"E k={k} tensor {i} round {rnd}"
+            assert_close_1e6(_np(gpu.theta_g[i]), orc.theta_g[i], f"theta_g {i} round {rnd}")
+            assert_close_1e6(_np(gpu.outer_u[i]), orc.outer_u[i], f"u {i} round {rnd}")
+            for k in range(K):
+                assert np.array_equal(_np(gpu.theta_k[k][i]), _np(gpu.theta_g[i]))
+            orc.theta_g[i][...] = _np(gpu.theta_g[i]); orc.outer_u[i][...] = _np(gpu.outer_u[i])
+    gpu.close()
+
+
+def test_two_stage_pseudogradient_is_bit_exact():
+    # eta_out = 1, mu = 0, u = 0: theta_new = theta - Psi, so Psi can be read back from the update
+    # (up to the one rounding of the subtraction) and compared with the oracle's codes
+    import dataclasses
+    import torch
+    w = dataclasses.replace(_sync_workload(4, 4, [(64, 256)]), quant_stages=2, outer_lr=1.0, outer_momentum=0.0)
+    rng = np.random.default_rng(9)
+    init = [np.zeros((64, 256), dtype=np.float32)]
+    gpu = gpu_for(w, init)
+    ths = [(0.05 * rng.standard_normal((64, 256))).astype(np.float32) for _ in range(4)]
+    for k in range(4):
+        gpu.theta_k[k][0].copy_(torch.from_numpy(ths[k]).cuda())
+    gpu.outer_sync(-1)
+    gpu.sync_status()
+    psi = O.compressed_pseudogradient(init[0], ths, 4, 128)
+    assert np.array_equal(_np(gpu.outer_u[0]), psi)        # u = 0 * u + 1 * Psi exactly
+    assert np.array_equal(_np(gpu.theta_g[0]), -psi)
+    gpu.close()
+
+
+def test_quantize_two_bits_vs_oracle(ns_ctx):
+    import torch
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((9, 300)).astype(np.float32)
+    codes, scales, deq = ns_ctx.quantize(torch.from_numpy(x).cuda(), 2)
+    rc, rs, rd = O.quantize_blocks(x, 2, 128)
+    assert np.array_equal(_np(codes), rc) and np.array_equal(_np(scales), rs) and np.array_equal(_np(deq), rd)
+    assert set(np.unique(rc)) <= {-1, 0, 1}
+
+
+def test_error_feedback_argument_errors():
+    import dataclasses
+    from paper_2505_23725_b200 import binding
+    w = dataclasses.replace(_sync_workload(2, 4, [(8, 128)]), quant_stages=1, error_feedback=True)
+    with pytest.raises(binding.MulocoError) as e:
+        gpu_for(w, [np.zeros((8, 128), np.float32)])
+    assert e.value.status == binding.EINVAL
