@@ -229,6 +229,9 @@ def main():
     ap.add_argument("--sync-only", type=int, nargs=3, metavar=("K", "MPARAMS", "QUANT"), default=None,
                     help="kernel study: time muloco_outer_sync on MPARAMS million parameters, K replicas, "
                          "QUANT in {0, 4, 8}")
+    ap.add_argument("--quant-stages", type=int, default=1, help="with --sync-only: 2 = per-worker quantisation + "
+                    "second quantisation of the mean (Algorithm 2)")
+    ap.add_argument("--ef", action="store_true", help="with --sync-only --quant-stages 2: error feedback")
     ap.add_argument("--adamw-only", type=int, nargs=2, metavar=("K", "MPARAMS"), default=None,
                     help="kernel study: time the AdamW part of muloco_inner_step on MPARAMS million parameters")
     ap.add_argument("--muon-only", type=int, nargs=4, metavar=("K", "LAYERS", "D", "F"), default=None,
@@ -474,7 +477,8 @@ def run_elementwise_only(args):
     rows = max(1, mparams * 1000000 // (8 * 4096))
     ts = [configs.Tensor(f"t{i}", rows, 4096, configs.ADAMW, 0) for i in range(8)]
     w = configs.Workload("elementwise-only", K=K, H=1, J=1, tensors=ts, muon_lr=0.02, muon_beta=0.9, muon_wd=0.01,
-                         outer_lr=0.7, outer_momentum=0.9, quant_bits=quant)
+                         outer_lr=0.7, outer_momentum=0.9, quant_bits=quant,
+                         quant_stages=args.quant_stages if sync else 1, error_feedback=bool(args.ef and sync))
     opt = binding.MuLoCo(w, "cuda:0", init_seed=1, alloc_grads=not sync)
     gen = torch.Generator(device="cuda"); gen.manual_seed(0)
     if sync:
@@ -498,7 +502,7 @@ def run_elementwise_only(args):
     n = w.n_params
     if sync:
         ms = ph["sync"] / args.steps
-        nbytes = n * (8.0 * K + 16.0)
+        nbytes = n * ((16.0 if args.ef else 8.0) * K + 16.0)      # error feedback: K more reads and writes
     else:
         ms = ph["adamw"] / args.steps
         nbytes = n * K * 28.0
