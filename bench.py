@@ -221,6 +221,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours")
+    ap.add_argument("--inner", default="muon", choices=["muon", "adamw"],
+                    help="adamw: the DiLoCo baseline (AdamW on every tensor) instead of MuLoCo")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workspace-gb", type=float, default=0.0)
@@ -250,6 +252,8 @@ def main():
 
     from paper_2505_23725_b200 import configs
     w = configs.workload(args.config)
+    if args.inner == "adamw":
+        w = configs.diloco_baseline(w)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -325,34 +329,43 @@ def main():
     # ---- roofline of the dominant kernel (Newton-Schulz tensor-core GEMMs) ----------------
     peaks = load_peaks()
     inner_steps = args.steps * w.H
-    ns_ms_per_inner = phases["ns"] / inner_steps
-    ns_tflops = w.ns_flops_credited() / (ns_ms_per_inner * 1e-3) / 1e12
-    peak_tf = peaks["bf16_tflops_sustained"]
-    ns_launches_per_inner = phases_launches_ns(w, opt)
-    shape_key = None
-    for tn in w.tensors:
-        if tn.name.endswith(".w1"):
-            shape_key = (tn.rows, tn.cols)
-            break
-    per_param = NS_TRAFFIC_BYTES_PER_PARAM.get(shape_key)
-    traffic = (per_param * w.n_muon_params * w.K / ns_launches_per_inner) if per_param else None
-    roofline = {"bound": "tensor", "kernel": "ns_tc_kernel (Gram / polynomial / apply GEMMs of Newton-Schulz)",
-                "achieved": ns_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": ns_tflops / peak_tf,
-                "peak_source": f"{peaks['source']} sustained bf16 matmul (kernel timed inside a long step)",
-                "launches_per_inner_step": ns_launches_per_inner,
-                "traffic": traffic, "traffic_unit": "bytes per launch (average over the launches of an inner step)",
-                "flops_convention": "credited 5*(4 s^2 l + 2 s^3) per matrix; symmetric products run upper-triangle tiles only",
-                "ms_per_inner_step": ns_ms_per_inner}
-    n_sync_rounds = args.steps
-    sync_gbs = w.sync_bytes() * n_sync_rounds / (phases["sync"] * 1e-3) / 1e9 if phases["sync"] > 0 else None
     n_adam = w.n_params - w.n_muon_params
     adam_bytes = n_adam * w.K * (28.0 if w.grad_dtype == "f32" else 26.0) * inner_steps
+    if w.n_muon_params > 0:
+        ns_ms_per_inner = phases["ns"] / inner_steps
+        ns_tflops = w.ns_flops_credited() / (ns_ms_per_inner * 1e-3) / 1e12
+        peak_tf = peaks["bf16_tflops_sustained"]
+        ns_launches_per_inner = phases_launches_ns(w, opt)
+        shape_key = None
+        for tn in w.tensors:
+            if tn.name.endswith(".w1"):
+                shape_key = (tn.rows, tn.cols)
+                break
+        per_param = NS_TRAFFIC_BYTES_PER_PARAM.get(shape_key)
+        traffic = (per_param * w.n_muon_params * w.K / ns_launches_per_inner) if per_param else None
+        roofline = {"bound": "tensor", "kernel": "ns_tc_kernel (Gram / polynomial / apply GEMMs of Newton-Schulz)",
+                    "achieved": ns_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": ns_tflops / peak_tf,
+                    "peak_source": f"{peaks['source']} sustained bf16 matmul (kernel timed inside a long step)",
+                    "launches_per_inner_step": ns_launches_per_inner,
+                    "traffic": traffic, "traffic_unit": "bytes per launch (average over the launches of an inner step)",
+                    "flops_convention": "credited 5*(4 s^2 l + 2 s^3) per matrix; symmetric products run upper-triangle tiles only",
+                    "ms_per_inner_step": ns_ms_per_inner}
+    else:
+        # DiLoCo baseline: the inner step is the AdamW kernel alone (HBM-bound)
+        ns_tflops = None
+        gbs = adam_bytes / (phases["adamw"] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "adamw_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} copy bandwidth",
+                    "traffic": adam_bytes / inner_steps, "traffic_unit": "bytes per launch (= algorithmic, see profiles/)"}
+    n_sync_rounds = args.steps
+    sync_gbs = w.sync_bytes() * n_sync_rounds / (phases["sync"] * 1e-3) / 1e9 if phases["sync"] > 0 else None
     adam_gbs = adam_bytes / (phases["adamw"] * 1e-3) / 1e9 if phases["adamw"] > 0 else None
     pro_bytes = w.n_muon_params * w.K * (14.0 if w.grad_dtype == "f32" else 12.0) * inner_steps
     pro_gbs = pro_bytes / (phases["prologue"] * 1e-3) / 1e9 if phases["prologue"] > 0 else None
     phase_report = {
         "ms_per_round": {k: v / args.steps for k, v in phases.items()},
-        "ns_tflops_credited": ns_tflops, "ns_frac_of_burst_peak": ns_tflops / peaks["bf16_tflops"],
+        "ns_tflops_credited": ns_tflops,
+        "ns_frac_of_burst_peak": (ns_tflops / peaks["bf16_tflops"]) if ns_tflops else None,
         "sync_gbs": sync_gbs, "sync_frac_of_hbm": (sync_gbs / peaks["hbm_gbs"]) if sync_gbs else None,
         "adamw_gbs": adam_gbs, "adamw_frac_of_hbm": (adam_gbs / peaks["hbm_gbs"]) if adam_gbs else None,
         "prologue_gbs": pro_gbs, "hbm_peak_gbs": peaks["hbm_gbs"],

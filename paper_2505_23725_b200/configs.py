@@ -134,6 +134,14 @@ def workload(idx: int) -> Workload:
     raise ValueError("workload index must be 0..4")
 
 
+def diloco_baseline(w: Workload) -> Workload:
+    """The DiLoCo baseline of the paper's comparisons: the same workload with AdamW as the inner
+    optimizer of EVERY tensor (Section 5, "DiLoCo"), outer step unchanged."""
+    import dataclasses
+    ts = [dataclasses.replace(t, kind=ADAMW) for t in w.tensors]
+    return dataclasses.replace(w, tensors=ts, name=w.name + "-diloco")
+
+
 def mini_workload(K=2, H=2, J=1, quant_bits=0, ns_mode="fp32", L=2, d=128, F=352,
                   vocab=0, norms=False, **kw) -> Workload:
     """A small custom workload for tests."""

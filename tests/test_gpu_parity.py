@@ -443,3 +443,28 @@ def test_error_feedback_argument_errors():
     with pytest.raises(binding.MulocoError) as e:
         gpu_for(w, [np.zeros((8, 128), np.float32)])
     assert e.value.status == binding.EINVAL
+
+
+def test_diloco_baseline_adamw_on_every_tensor():
+    # the paper's DiLoCo comparison: same round, AdamW as the inner optimizer of every tensor
+    w = configs.diloco_baseline(configs.mini_workload(K=2, H=2, L=1, d=64, F=96, vocab=50, norms=True))
+    assert all(t.kind == configs.ADAMW for t in w.tensors)
+    rng = np.random.default_rng(33)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init)
+    for h in range(w.H):
+        gs = [synth.host_gradients(rng, w.tensors) for _ in range(w.K)]
+        gpu.inner_step(-1, to_dev(gs))
+        orc.inner_step_all(gs)
+    gpu.sync_status()
+    for k in range(w.K):
+        for i in range(gpu.n):
+            assert_close_1e6(_np(gpu.theta_k[k][i]), orc.theta_k[k][i], f"theta k={k} i={i}")
+            orc.theta_k[k][i][...] = _np(gpu.theta_k[k][i])
+    gpu.outer_sync(-1)
+    orc.outer_sync(-1)
+    gpu.sync_status()
+    for i in range(gpu.n):
+        assert_close_1e6(_np(gpu.theta_g[i]), orc.theta_g[i], f"theta_g {i}")
+    gpu.close()
