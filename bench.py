@@ -292,7 +292,10 @@ def main():
             t += 1
             for f in opt.fragments_due(t):
                 opt.outer_sync(f)
+                sync_calls[0] += 1
         return t
+
+    sync_calls = [0]
 
     def barrier():
         if distributed:
@@ -305,6 +308,7 @@ def main():
     opt.sync_status()
     opt.set_timing(True)
     opt.get_timings()
+    sync_calls[0] = 0
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
@@ -335,7 +339,7 @@ def main():
         ns_ms_per_inner = phases["ns"] / inner_steps
         ns_tflops = w.ns_flops_credited() / (ns_ms_per_inner * 1e-3) / 1e12
         peak_tf = peaks["bf16_tflops_sustained"]
-        ns_launches_per_inner = phases_launches_ns(w, opt)
+        ns_launches_per_inner = ns_launches_per_inner_step(launches, sync_calls[0], inner_steps, n_adam > 0)
         shape_key = None
         for tn in w.tensors:
             if tn.name.endswith(".w1"):
@@ -394,21 +398,11 @@ def main():
         dist.destroy_process_group()
 
 
-def phases_launches_ns(w, opt):
-    """Newton-Schulz GEMM launches per inner step: 15 per chunk of every shape group."""
-    ph, n = 0, 0
-    groups = {}
-    for t in w.tensors:
-        if t.kind == "muon":
-            key = (min(t.rows, t.cols), max(t.rows, t.cols))
-            groups[key] = groups.get(key, 0) + w.K
-    budget = opt.cfg.workspace_bytes or (6 << 30)
-    for (s_, l_), count in groups.items():
-        ldx, lds = (l_ + 7) // 8 * 8, (s_ + 7) // 8 * 8
-        per = 2 * s_ * ldx * 2 + 2 * s_ * lds * 2
-        ch = max(1, min(count, budget // per))
-        n += 15 * ((count + ch - 1) // ch)
-    return n
+def ns_launches_per_inner_step(total_launches, sync_launches, inner_steps, has_adamw):
+    """Newton-Schulz GEMM launches per inner step, from the library's own launch counter: an inner
+    step launches, per workspace chunk, 2 prologue kernels and 15 GEMM kernels, plus one AdamW kernel."""
+    per_inner = (total_launches - sync_launches) / inner_steps - (1 if has_adamw else 0)
+    return int(round(per_inner / 17.0 * 15.0))
 
 
 def run_ns_only(args):

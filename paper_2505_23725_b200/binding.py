@@ -200,8 +200,13 @@ class MuLoCo:
         self.flat_u = torch.zeros(off, dtype=f32, device=dev)
         self.flat_theta_k = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)]
         self.flat_s1 = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)]
-        self.flat_s2 = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)] \
-            if any(t.kind == _cfg.ADAMW for t in workload.tensors) else [None] * self.K
+        # Adam's second moment exists for AdamW tensors only: its own compact buffer
+        self.offsets2, off2 = [], 0
+        for t in workload.tensors:
+            self.offsets2.append(off2 if t.kind == _cfg.ADAMW else None)
+            if t.kind == _cfg.ADAMW:
+                off2 += (t.numel + self.ALIGN - 1) // self.ALIGN * self.ALIGN
+        self.flat_s2 = [torch.empty(off2, dtype=f32, device=dev) if off2 else None for _ in range(self.K)]
         self.flat_ef = [torch.empty(off, dtype=f32, device=dev) for _ in range(self.K)] \
             if workload.error_feedback else None
         self.ef = [self._views(b) for b in self.flat_ef] if self.flat_ef else None
@@ -209,7 +214,8 @@ class MuLoCo:
         self.outer_u = self._views(self.flat_u)
         self.theta_k = [self._views(b) for b in self.flat_theta_k]
         self.state1 = [self._views(b) for b in self.flat_s1]
-        self.state2 = [self._views(b) if b is not None else [None] * self.n for b in self.flat_s2]
+        self.state2 = [[b[o:o + t.numel].view(t.rows, t.cols) if (b is not None and o is not None) else None
+                        for o, t in zip(self.offsets2, workload.tensors)] for b in self.flat_s2]
         if init is not None:
             for i, a in enumerate(init):
                 self.theta_g[i].copy_(torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev))

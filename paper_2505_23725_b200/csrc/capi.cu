@@ -444,7 +444,14 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
     c->groups[gidx[key]].tensors.push_back(i);
   }
   const int elt = (cfg->ns_mode == MULOCO_NS_BF16) ? 2 : 4;
-  const size_t budget = cfg->workspace_bytes ? (size_t)cfg->workspace_bytes : ((size_t)6 << 30);
+  // default budget: 6 GiB, less when the device is nearly full (the state of the largest
+  // configurations leaves only a few GiB)
+  size_t budget = cfg->workspace_bytes ? (size_t)cfg->workspace_bytes : ((size_t)6 << 30);
+  if (!cfg->workspace_bytes) {
+    size_t free_b = 0, total_b = 0;
+    if (cudaMemGetInfo(&free_b, &total_b) == cudaSuccess && free_b / 2 < budget)
+      budget = std::max<size_t>(free_b / 2, (size_t)256 << 20);
+  }
   size_t need = 0;
   for (Group& g : c->groups) {
     const int np = prologue_partials_per_matrix(g.s, g.l);

@@ -255,10 +255,12 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
     const int64_t base = (unit - s.unit_begin) * ADAM_UNIT;
     int64_t cnt = s.n - base;
     if (cnt > ADAM_UNIT) cnt = ADAM_UNIT;
-    const bool vec = !g_is_bf16 &&
-                     ((((uintptr_t)s.g | (uintptr_t)s.m | (uintptr_t)s.v | (uintptr_t)s.theta) & 15) == 0);
+    // 16-byte accesses when every stream allows it (bf16 gradients: 8 bytes for the same 4 elements)
+    const bool vec = ((((uintptr_t)s.m | (uintptr_t)s.v | (uintptr_t)s.theta) & 15) == 0) &&
+                     ((((uintptr_t)s.g) & (g_is_bf16 ? 7 : 15)) == 0);
     if (vec) {
       const float4* g4 = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(s.g) + base);
+      const uint2* gb = reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(s.g) + base);
       float4* m4 = reinterpret_cast<float4*>(s.m + base);
       float4* v4 = reinterpret_cast<float4*>(s.v + base);
       float4* t4 = reinterpret_cast<float4*>(s.theta + base);
@@ -267,7 +269,14 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
       for (int r = 0; r < ADAM_UNIT / 4 / ADAM_THREADS; ++r) {
         const int i = threadIdx.x + r * ADAM_THREADS;
         if (i < n4) {
-          const float4 g = __ldcs(g4 + i);
+          float4 g;
+          if (g_is_bf16) {
+            const uint2 raw = __ldcs(gb + i);
+            g = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                            __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+          } else {
+            g = __ldcs(g4 + i);
+          }
           float4 m = m4[i], v = v4[i], t = t4[i];
           adam_elem(g.x, m.x, v.x, t.x, beta1, beta2, eps, s);
           adam_elem(g.y, m.y, v.y, t.y, beta1, beta2, eps, s);
@@ -277,7 +286,7 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
         }
       }
       for (int64_t i = (int64_t)n4 * 4 + threadIdx.x; i < cnt; i += ADAM_THREADS) {
-        float g = reinterpret_cast<const float*>(s.g)[base + i];
+        float g = load_g(s.g, base + i, g_is_bf16);
         float m = s.m[base + i], v = s.v[base + i], t = s.theta[base + i];
         adam_elem(g, m, v, t, beta1, beta2, eps, s);
         s.m[base + i] = m; s.v[base + i] = v; s.theta[base + i] = t;
