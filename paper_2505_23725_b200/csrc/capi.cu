@@ -114,7 +114,12 @@ struct muloco_ctx {
 
   std::vector<int64_t> worker_step, frag_syncs;
 
-  // host-gradient staging
+  // host-gradient staging: copies run on their own stream, one section (shape group, or the
+  // AdamW tensors) at a time, so that the copy of a section overlaps the compute of the others
+  cudaStream_t copy_st = nullptr;
+  std::vector<cudaEvent_t> ev_copied, ev_consumed;   // per section
+  std::vector<char> consumed_valid;
+  bool host_mode = false;                            // set while muloco_inner_step_host runs the step
   char* stage = nullptr;
   size_t stage_bytes = 0;
   std::vector<size_t> stage_off;   // [K][n]
@@ -160,17 +165,19 @@ struct PhaseTimer {
   muloco_ctx* c;
   TimedSpan sp;
   bool on;
-  PhaseTimer(muloco_ctx* ctx, int phase) : c(ctx), on(ctx->timing) {
+  cudaStream_t stream;
+  PhaseTimer(muloco_ctx* ctx, int phase, cudaStream_t s = nullptr)
+      : c(ctx), on(ctx->timing), stream(s ? s : ctx->st) {
     if (on) {
       sp.phase = phase;
       sp.a = get_event(c);
       sp.b = get_event(c);
-      cudaEventRecord(sp.a, c->st);
+      cudaEventRecord(sp.a, stream);
     }
   }
   ~PhaseTimer() {
     if (on) {
-      cudaEventRecord(sp.b, c->st);
+      cudaEventRecord(sp.b, stream);
       c->spans.push_back(sp);
     }
   }
@@ -531,6 +538,10 @@ MULOCO_API void muloco_destroy(muloco_ctx* c) {
   if (c->d_mats) cudaFree(c->d_mats);
   if (c->d_adam) cudaFree(c->d_adam);
   if (c->d_wmaps) cudaFree(c->d_wmaps);
+  if (c->copy_st) cudaStreamSynchronize(c->copy_st);
+  for (cudaEvent_t e : c->ev_copied) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ev_consumed) if (e) cudaEventDestroy(e);
+  if (c->copy_st) cudaStreamDestroy(c->copy_st);
   if (c->stage) cudaFree(c->stage);
   for (FragTable& f : c->frags)
     if (f.d_segs) cudaFree(f.d_segs);
@@ -616,17 +627,30 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
   for (size_t gi = 0; gi < c->groups.size(); ++gi) {
     Group& g = c->groups[gi];
     const int count = (int)g.tensors.size() * nw;
+    if (c->host_mode) CK(cudaStreamWaitEvent(c->st, c->ev_copied[gi], 0));
     for (int m0 = 0; m0 < count; m0 += g.chunk) {
       const int cnt = std::min(g.chunk, count - m0);
       rs = run_ns_chunk(c, g, c->ws, c->d_mats + group_begin[gi] + m0, cnt, f.ns_mode, SRC_MUON,
                         SINK_UPDATE_W, g_is_bf16);
       if (rs != MULOCO_OK) return rs;
     }
+    if (c->host_mode) {
+      CK(cudaEventRecord(c->ev_consumed[gi], c->st));
+      c->consumed_valid[gi] = 1;
+    }
   }
   if (na) {
-    PhaseTimer t(c, MULOCO_PH_ADAMW);
-    launch_adamw(c->st, c->d_adam, (int)na, units, g_is_bf16, f.adam_beta1, f.adam_beta2, f.adam_eps);
-    c->launches += 1;
+    const size_t sec = c->groups.size();
+    if (c->host_mode) CK(cudaStreamWaitEvent(c->st, c->ev_copied[sec], 0));
+    {
+      PhaseTimer t(c, MULOCO_PH_ADAMW);
+      launch_adamw(c->st, c->d_adam, (int)na, units, g_is_bf16, f.adam_beta1, f.adam_beta2, f.adam_eps);
+      c->launches += 1;
+    }
+    if (c->host_mode) {
+      CK(cudaEventRecord(c->ev_consumed[sec], c->st));
+      c->consumed_valid[sec] = 1;
+    }
   }
   CK(cudaGetLastError());
   return MULOCO_OK;
@@ -654,20 +678,43 @@ MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* c, int32_t worker, c
   }
   const int k0 = worker < 0 ? 0 : worker, k1 = worker < 0 ? K : worker + 1;
   std::vector<const void*> dev((size_t)(k1 - k0) * n);
-  {
-    PhaseTimer t(c, MULOCO_PH_COPY);
-    // one copy per tensor: adjacent host pointers may still belong to different
-    // pinned allocations, which a single copy must not span
-    for (int k = k0; k < k1; ++k)
-      for (int i = 0; i < n; ++i) {
-        const void* src = host_grads[(size_t)(k - k0) * n + i];
-        if (!src) return fail(c, MULOCO_EINVAL, "host gradient of tensor %d (worker %d) is NULL", i, k);
-        char* dst = c->stage + c->stage_off[(size_t)k * n + i];
-        dev[(size_t)(k - k0) * n + i] = dst;
-        CK(cudaMemcpyAsync(dst, src, (size_t)c->T[i].numel() * elt, cudaMemcpyHostToDevice, c->st));
-      }
+  for (int k = k0; k < k1; ++k)
+    for (int i = 0; i < n; ++i)
+      if (!host_grads[(size_t)(k - k0) * n + i])
+        return fail(c, MULOCO_EINVAL, "host gradient of tensor %d (worker %d) is NULL", i, k);
+  const size_t n_sec = c->groups.size() + 1;           // shape groups, then the AdamW tensors
+  if (!c->copy_st) {
+    CK(cudaStreamCreateWithFlags(&c->copy_st, cudaStreamNonBlocking));
+    c->ev_copied.assign(n_sec, nullptr);
+    c->ev_consumed.assign(n_sec, nullptr);
+    c->consumed_valid.assign(n_sec, 0);
+    for (size_t s2 = 0; s2 < n_sec; ++s2) {
+      CK(cudaEventCreateWithFlags(&c->ev_copied[s2], cudaEventDisableTiming));
+      CK(cudaEventCreateWithFlags(&c->ev_consumed[s2], cudaEventDisableTiming));
+    }
   }
-  return muloco_inner_step(c, worker, dev.data(), lr_scale);
+  // Section by section, in the order the step consumes them: wait until the previous step has
+  // consumed the section's staging area, copy (one copy per tensor: adjacent host pointers may
+  // belong to different pinned allocations, which a single copy must not span), signal.
+  for (size_t sec = 0; sec < n_sec; ++sec) {
+    const std::vector<int>& ids = sec < c->groups.size() ? c->groups[sec].tensors : c->adam_ids;
+    if (c->consumed_valid[sec]) CK(cudaStreamWaitEvent(c->copy_st, c->ev_consumed[sec], 0));
+    {
+      PhaseTimer t(c, MULOCO_PH_COPY, c->copy_st);
+      for (int k = k0; k < k1; ++k)
+        for (int i : ids) {
+          const void* src = host_grads[(size_t)(k - k0) * n + i];
+          char* dst = c->stage + c->stage_off[(size_t)k * n + i];
+          dev[(size_t)(k - k0) * n + i] = dst;
+          CK(cudaMemcpyAsync(dst, src, (size_t)c->T[i].numel() * elt, cudaMemcpyHostToDevice, c->copy_st));
+        }
+    }
+    CK(cudaEventRecord(c->ev_copied[sec], c->copy_st));
+  }
+  c->host_mode = true;
+  const muloco_status rs = muloco_inner_step(c, worker, dev.data(), lr_scale);
+  c->host_mode = false;
+  return rs;
 }
 
 MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* c, int32_t fragment) {
