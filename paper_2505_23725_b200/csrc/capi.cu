@@ -761,8 +761,9 @@ MULOCO_API int32_t muloco_fragments_due(const muloco_ctx* c, int64_t step, int32
 MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* c, const void* X, int32_t x_dtype, void* O, int32_t o_dtype,
                                    int32_t batch, int64_t rows, int64_t cols, int32_t ns_mode) {
   if (!c) return MULOCO_EINVAL;
-  if (!X || !O) return fail(c, MULOCO_EINVAL, "X or O is NULL");
   if (batch < 0 || rows < 1 || cols < 1) return fail(c, MULOCO_ESHAPE, "bad batch/shape");
+  if (batch == 0) return MULOCO_OK;                  // an empty batch: nothing to read or write
+  if (!X || !O) return fail(c, MULOCO_EINVAL, "X or O is NULL");
   if ((x_dtype != MULOCO_F32 && x_dtype != MULOCO_BF16) || (o_dtype != MULOCO_F32 && o_dtype != MULOCO_BF16))
     return fail(c, MULOCO_EINVAL, "bad dtype");
   if (ns_mode != MULOCO_NS_BF16 && ns_mode != MULOCO_NS_FP32) return fail(c, MULOCO_EINVAL, "bad ns_mode");
@@ -829,10 +830,10 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* c, const void* X, int3
 MULOCO_API muloco_status muloco_quantize(muloco_ctx* c, const float* psi, int64_t rows, int64_t cols, int32_t bits,
                               int8_t* codes, float* scales, float* dequant) {
   if (!c) return MULOCO_EINVAL;
-  if (!psi) return fail(c, MULOCO_EINVAL, "psi is NULL");
   if (bits != 8 && bits != 4 && bits != 2) return fail(c, MULOCO_EINVAL, "bits must be 8, 4 or 2");
   if (rows < 0 || cols < 0) return fail(c, MULOCO_ESHAPE, "negative shape");
-  if (rows == 0 || cols == 0) return MULOCO_OK;
+  if (rows == 0 || cols == 0) return MULOCO_OK;      // empty input: nothing to read or write
+  if (!psi) return fail(c, MULOCO_EINVAL, "psi is NULL");
   launch_quantize(c->st, psi, rows, cols, c->cfg.quant_block, bits, codes, scales, dequant, c->d_status);
   c->launches += 1;
   CK(cudaGetLastError());
