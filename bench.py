@@ -233,6 +233,7 @@ def main():
                          "QUANT in {0, 4, 8}")
     ap.add_argument("--quant-stages", type=int, default=1, help="with --sync-only: 2 = per-worker quantisation + "
                     "second quantisation of the mean (Algorithm 2)")
+    ap.add_argument("--quant-block", type=int, default=128, help="with --sync-only: 32/64/128, or 0 = row-wise")
     ap.add_argument("--ef", action="store_true", help="with --sync-only --quant-stages 2: error feedback")
     ap.add_argument("--adamw-only", type=int, nargs=2, metavar=("K", "MPARAMS"), default=None,
                     help="kernel study: time the AdamW part of muloco_inner_step on MPARAMS million parameters")
@@ -485,7 +486,8 @@ def run_elementwise_only(args):
     ts = [configs.Tensor(f"t{i}", rows, 4096, configs.ADAMW, 0) for i in range(8)]
     w = configs.Workload("elementwise-only", K=K, H=1, J=1, tensors=ts, muon_lr=0.02, muon_beta=0.9, muon_wd=0.01,
                          outer_lr=0.7, outer_momentum=0.9, quant_bits=quant,
-                         quant_stages=args.quant_stages if sync else 1, error_feedback=bool(args.ef and sync))
+                         quant_stages=args.quant_stages if sync else 1, error_feedback=bool(args.ef and sync),
+                         quant_block=args.quant_block)
     opt = binding.MuLoCo(w, "cuda:0", init_seed=1, alloc_grads=not sync)
     gen = torch.Generator(device="cuda"); gen.manual_seed(0)
     if sync:

@@ -85,7 +85,9 @@ typedef struct {
   int32_t adam_bias_correction; /* 1: divide by 1 - beta^t                              */
   float outer_lr, outer_momentum; /* eta_out, mu of Eq. (3)                             */
   int32_t quant;       /* muloco_quant: quantise -> dequantise the pseudogradient       */
-  int32_t quant_block; /* elements per absmax block along a row (128)                   */
+  int32_t quant_block; /* elements per absmax block along a row (32, 64 or 128), or 0 for
+                          row-wise quantisation: one block per row (rows of up to ~50,000
+                          elements; longer rows make muloco_outer_sync return MULOCO_ESHAPE) */
   int32_t grad_dtype;  /* muloco_dtype of the gradients given to muloco_inner_step      */
   int32_t quant_stages; /* 0 or 1: quantise the averaged pseudogradient once (benchmark form);
                            2: Algorithm 2 with the two quantisations of Section 2

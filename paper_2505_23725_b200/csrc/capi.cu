@@ -48,6 +48,7 @@ struct FragTable {
   SyncSeg* d_segs = nullptr;
   int n_segs = 0;
   int64_t n_units = 0;
+  int64_t max_cols = 0;
   std::vector<int> tensors;
 };
 
@@ -183,7 +184,7 @@ struct PhaseTimer {
   }
 };
 
-bool valid_block(int b) { return b == 32 || b == 64 || b == 128; }
+bool valid_block(int b) { return b == 0 || b == 32 || b == 64 || b == 128; }   // 0: one block per row
 
 muloco_status validate_config(const muloco_config* cfg) {
   muloco_ctx* c = nullptr;
@@ -204,7 +205,7 @@ muloco_status validate_config(const muloco_config* cfg) {
     return fail(c, MULOCO_EINVAL, "error_feedback needs quant_stages == 2 and a quantiser");
   if (cfg->error_feedback != 0 && !(cfg->ef_beta >= 0.f && cfg->ef_beta <= 1.f))
     return fail(c, MULOCO_EINVAL, "ef_beta must be in [0, 1]");
-  if (!valid_block(cfg->quant_block)) return fail(c, MULOCO_EINVAL, "quant_block must be 32, 64 or 128");
+  if (!valid_block(cfg->quant_block)) return fail(c, MULOCO_EINVAL, "quant_block must be 0 (row-wise), 32, 64 or 128");
   if (cfg->grad_dtype != MULOCO_F32 && cfg->grad_dtype != MULOCO_BF16)
     return fail(c, MULOCO_EINVAL, "unknown grad_dtype %d", cfg->grad_dtype);
   if (!(cfg->ns_eps >= 0.f)) return fail(c, MULOCO_EINVAL, "ns_eps must be >= 0");
@@ -314,8 +315,10 @@ muloco_status build_sync_tables(muloco_ctx* c) {
       s.theta_g = t.theta_g; s.u = t.u;
       if (c->cfg.quant == MULOCO_Q_NONE) { s.rows = 1; s.cols = t.numel(); }
       else { s.rows = t.rows; s.cols = t.cols; }
-      const int64_t blk = (c->cfg.quant == MULOCO_Q_NONE) ? 128 : c->cfg.quant_block;
+      int64_t blk = (c->cfg.quant == MULOCO_Q_NONE) ? 128 : c->cfg.quant_block;
+      if (blk == 0) blk = s.cols;                      // row-wise: one unit per row
       s.nblk = (s.cols + blk - 1) / blk;
+      ft.max_cols = std::max<int64_t>(ft.max_cols, s.cols);
       s.unit_begin = units;
       s.rep_index = (int64_t)i * K;
       units += s.rows * s.nblk;
@@ -726,6 +729,17 @@ MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* c, int32_t fragment) {
   if (ft.n_segs == 0) return MULOCO_OK;
   PhaseTimer t(c, MULOCO_PH_SYNC);
   const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
+  if (f.quant != MULOCO_Q_NONE && blk == 0) {
+    cudaError_t e = launch_outer_sync_rows(c->st, ft.d_segs, ft.n_segs, c->d_replicas, f.K, ft.n_units, ft.max_cols,
+                                           f.quant, f.outer_lr, f.outer_momentum, c->d_status,
+                                           f.quant_stages == 2 ? 2 : 1, c->d_ef, f.ef_beta);
+    if (e == cudaErrorInvalidValue)
+      return fail(c, MULOCO_ESHAPE, "row-wise quantisation: a row of %lld elements does not fit shared memory",
+                  (long long)ft.max_cols);
+    CK(e);
+    c->launches += 1;
+    return MULOCO_OK;
+  }
   launch_outer_sync(c->st, ft.d_segs, ft.n_segs, c->d_replicas, f.K, ft.n_units, blk, f.quant, f.outer_lr,
                     f.outer_momentum, c->d_status, c->n_sms, f.quant_stages == 2 ? 2 : 1, c->d_ef, f.ef_beta);
   c->launches += 1;
@@ -833,6 +847,8 @@ MULOCO_API muloco_status muloco_quantize(muloco_ctx* c, const float* psi, int64_
   if (bits != 8 && bits != 4 && bits != 2) return fail(c, MULOCO_EINVAL, "bits must be 8, 4 or 2");
   if (rows < 0 || cols < 0) return fail(c, MULOCO_ESHAPE, "negative shape");
   if (rows == 0 || cols == 0) return MULOCO_OK;      // empty input: nothing to read or write
+  if (c->cfg.quant_block == 0)
+    return fail(c, MULOCO_ESHAPE, "muloco_quantize works on blocks of 32, 64 or 128; this context is row-wise");
   if (!psi) return fail(c, MULOCO_EINVAL, "psi is NULL");
   launch_quantize(c->st, psi, rows, cols, c->cfg.quant_block, bits, codes, scales, dequant, c->d_status);
   c->launches += 1;

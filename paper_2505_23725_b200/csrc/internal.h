@@ -102,6 +102,11 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
                        int K, int64_t n_units, int block, int quant_bits, float outer_lr,
                        float mu, int* status, int n_sms, int stages = 1, float* const* ef = nullptr,
                        float ef_beta = 1.0f);
+// Row-wise quantisation (quant_block == 0): units are rows (SyncSeg.nblk == 1); max_cols is the
+// longest row of the fragment.  cudaErrorInvalidValue when a row does not fit shared memory.
+cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
+                                   int K, int64_t n_rows, int64_t max_cols, int quant_bits, float outer_lr,
+                                   float mu, int* status, int stages, float* const* ef, float ef_beta);
 void launch_pseudogradient(cudaStream_t st, const float* theta_g, float* const* replicas, int K,
                            int64_t n, float* psi_out);
 void launch_quantize(cudaStream_t st, const float* psi, int64_t rows, int64_t cols, int block,

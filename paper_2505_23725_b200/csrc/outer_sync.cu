@@ -299,6 +299,122 @@ outer_sync2_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* _
   if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
 }
 
+// Row-wise quantisation (one absmax block per row; Section 6.3 and the row-wise panels of the
+// quantisation ablation): one CTA per row.  The row's pseudogradient (or, with two stages, the mean
+// of the workers' dequantised deltas) is staged in shared memory between the pass that finds the
+// row's absmax and the pass that quantises it.  With two stages every replica is read twice: once
+// for its own absmax, once to be quantised with it.  Arithmetic and order are those of the block
+// kernels, so codes are bit-exact against the same reference.
+constexpr int ROW_THREADS = 256;
+
+__device__ __forceinline__ float block_max(float v, float* red) {
+  v = warp_max(v);
+  __syncthreads();                       // red may still be read from the previous reduction
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float m = red[0];
+#pragma unroll
+  for (int w = 1; w < ROW_THREADS / 32; ++w) m = fmaxf(m, red[w]);
+  return m;
+}
+
+template <int QB>
+__device__ __forceinline__ float quant_dequant1(float x, float amax, bool& bad) {
+  constexpr float qmax = (QB == 8) ? 127.0f : (QB == 4 ? 7.0f : 1.0f);
+  if (!(fabsf(x) <= FLT_MAX)) bad = true;
+  if (!(amax > 0.0f && amax <= FLT_MAX)) return 0.0f;
+  const float inv = __fdiv_rn(qmax, amax);
+  const float scale = __fdiv_rn(amax, qmax);
+  float r = rintf(__fmul_rn(x, inv));
+  r = fminf(fmaxf(r, -qmax), qmax);
+  return __fmul_rn(r, scale);
+}
+
+template <int QB, bool TWO, bool EF>
+__global__ void __launch_bounds__(ROW_THREADS)
+outer_sync_row_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps,
+                      float* const* __restrict__ efs, int K, int64_t n_rows, float eta, float mu, float inv_k,
+                      float ef_beta, int* __restrict__ status) {
+  extern __shared__ float rowbuf[];      // [cols] staged values, then [K] per-worker absmax
+  __shared__ float red[ROW_THREADS / 32];
+  const int64_t unit = blockIdx.x;
+  if (unit >= n_rows) return;
+  const int seg = find_seg(segs, n_segs, unit);
+  const SyncSeg s = segs[seg];
+  const int64_t row = unit - s.unit_begin;
+  const int64_t cols = s.cols;
+  const int64_t off0 = row * cols;
+  float* const* rp = reps + s.rep_index;
+  float* const* ep = EF ? efs + s.rep_index : nullptr;
+  float* amax_k = rowbuf + cols;
+  bool bad = false;
+  const float* tgp = s.theta_g + off0;
+
+  if (TWO) {
+    // pass A: every worker's absmax over the row
+    for (int k = 0; k < K; ++k) {
+      const float* r = rp[k] + off0;
+      const float* e = EF ? ep[k] + off0 : nullptr;
+      float lm = 0.f;
+      for (int64_t c = threadIdx.x; c < cols; c += ROW_THREADS) {
+        const float d = __fsub_rn(tgp[c], r[c]);
+        const float x = EF ? __fadd_rn(__fmul_rn(ef_beta, e[c]), d) : d;
+        const float a = fabsf(x);
+        if (!(a <= FLT_MAX)) bad = true;
+        lm = fmaxf(lm, a);
+      }
+      const float m = block_max(lm, red);
+      if (threadIdx.x == 0) amax_k[k] = m;
+    }
+    __syncthreads();
+    // pass B: quantise every worker's value with its own scale, mean in fp32, stage the mean
+    float lm = 0.f;
+    for (int64_t c = threadIdx.x; c < cols; c += ROW_THREADS) {
+      const float t = tgp[c];
+      float acc = 0.f;
+      for (int k = 0; k < K; ++k) {
+        const float d = __fsub_rn(t, rp[k][off0 + c]);
+        float x = d;
+        if (EF) x = __fadd_rn(__fmul_rn(ef_beta, ep[k][off0 + c]), d);
+        const float sent = quant_dequant1<QB>(x, amax_k[k], bad);
+        if (EF) ep[k][off0 + c] = __fsub_rn(x, sent);
+        acc = __fadd_rn(acc, sent);
+      }
+      const float mean = __fmul_rn(acc, inv_k);
+      rowbuf[c] = mean;
+      lm = fmaxf(lm, fabsf(mean));
+    }
+    const float amax = block_max(lm, red);
+    for (int64_t c = threadIdx.x; c < cols; c += ROW_THREADS) rowbuf[c] = quant_dequant1<QB>(rowbuf[c], amax, bad);
+  } else {
+    float lm = 0.f;
+    for (int64_t c = threadIdx.x; c < cols; c += ROW_THREADS) {
+      const float t = tgp[c];
+      float acc = 0.f;
+      for (int k = 0; k < K; ++k) acc = __fadd_rn(acc, __fsub_rn(t, rp[k][off0 + c]));
+      const float psi = __fmul_rn(acc, inv_k);
+      rowbuf[c] = psi;
+      const float a = fabsf(psi);
+      if (!(a <= FLT_MAX)) bad = true;
+      lm = fmaxf(lm, a);
+    }
+    const float amax = block_max(lm, red);
+    for (int64_t c = threadIdx.x; c < cols; c += ROW_THREADS) rowbuf[c] = quant_dequant1<QB>(rowbuf[c], amax, bad);
+  }
+  // each thread re-reads only the entries it wrote: no barrier needed before the update pass
+  for (int64_t c = threadIdx.x; c < cols; c += ROW_THREADS) {
+    const float psi = rowbuf[c];
+    const float t = tgp[c];
+    const float ep_ = eta * psi;
+    const float un = fmaf(mu, s.u[off0 + c], ep_);
+    const float tn = t - fmaf(mu, un, ep_);
+    s.u[off0 + c] = un;
+    s.theta_g[off0 + c] = tn;
+    for (int k = 0; k < K; ++k) rp[k][off0 + c] = tn;
+  }
+  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, ST_NONFINITE);
+}
+
 __global__ void pseudograd_kernel(const float* __restrict__ tg, float* const* __restrict__ reps, int K,
                                   int64_t n, float inv_k, float* __restrict__ out) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -406,6 +522,36 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
     launch_sync_q<2>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
   else
     launch_sync_q<0>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+}
+
+cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
+                                   int K, int64_t n_rows, int64_t max_cols, int quant_bits, float outer_lr,
+                                   float mu, int* status, int stages, float* const* ef, float ef_beta) {
+  if (n_rows <= 0) return cudaSuccess;
+  const size_t smem = ((size_t)max_cols + (size_t)K) * sizeof(float);
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  const float inv_k = 1.0f / (float)K;
+  const bool two = (stages == 2);
+#define MULOCO_ROW_LAUNCH(QB, TWO, EF)                                                                   \
+  do {                                                                                                   \
+    cudaError_t e_ = cudaFuncSetAttribute(outer_sync_row_kernel<QB, TWO, EF>,                            \
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024)); \
+    if (e_ != cudaSuccess) return e_;                                                                    \
+    outer_sync_row_kernel<QB, TWO, EF><<<(unsigned)n_rows, ROW_THREADS, smem, st>>>(                     \
+        segs, n_segs, replicas, ef, K, n_rows, outer_lr, mu, inv_k, ef_beta, status);                    \
+  } while (0)
+#define MULOCO_ROW_BITS(QB)                                   \
+  do {                                                        \
+    if (two && ef) MULOCO_ROW_LAUNCH(QB, true, true);         \
+    else if (two) MULOCO_ROW_LAUNCH(QB, true, false);         \
+    else MULOCO_ROW_LAUNCH(QB, false, false);                 \
+  } while (0)
+  if (quant_bits == 8) MULOCO_ROW_BITS(8);
+  else if (quant_bits == 4) MULOCO_ROW_BITS(4);
+  else MULOCO_ROW_BITS(2);
+#undef MULOCO_ROW_BITS
+#undef MULOCO_ROW_LAUNCH
+  return cudaGetLastError();
 }
 
 void launch_pseudogradient(cudaStream_t st, const float* theta_g, float* const* replicas, int K,

@@ -496,3 +496,53 @@ def test_one_by_n_and_n_by_one_matrices_through_newton_schulz(ns_ctx):
             assert relfro(out, ref) < tol, f"{shape} {mode}: {relfro(out, ref):.3e}"
             assert abs(np.linalg.norm(ref) - 0.696436) < 1e-4      # p applied five times to 1
     ns_ctx.sync_status()
+
+
+ROW_SHAPES = [(3, 5000), (4, 300), (1, 1000), (64, 128), (257, 131), (2, 7), (5, 32000)]
+
+
+@pytest.mark.parametrize("K", [1, 3, 8])
+@pytest.mark.parametrize("bits,stages,ef", [(8, 1, False), (4, 1, False), (4, 2, False), (2, 2, False), (8, 2, True),
+                                            (4, 2, True)])
+def test_row_wise_quantised_sync_vs_oracle(K, bits, stages, ef):
+    # one absmax block per row (quant_block = 0), single- and two-stage, with and without error feedback
+    import dataclasses
+    import torch
+    w = dataclasses.replace(_sync_workload(K, bits, ROW_SHAPES), quant_block=0, quant_stages=stages,
+                            error_feedback=ef, ef_beta=0.9)
+    rng = np.random.default_rng(900 + 10 * K + bits + stages + ef)
+    init = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) * 0.02 for t in w.tensors]
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init, quant_stages=stages, error_feedback=ef, ef_beta=0.9)
+    for rnd in range(2):
+        for k in range(K):
+            for i, t in enumerate(w.tensors):
+                drift = (rng.standard_normal((t.rows, t.cols)) * 10.0 ** rng.uniform(-4, -1)).astype(np.float32)
+                if i == 1 and rnd == 0:
+                    drift[2, :] = 0.0                      # a row whose pseudogradient is exactly zero
+                orc.theta_k[k][i][...] = orc.theta_g[i] + drift
+                gpu.theta_k[k][i].copy_(torch.from_numpy(orc.theta_k[k][i]).cuda())
+        gpu.outer_sync(-1)
+        orc.outer_sync(-1)
+        gpu.sync_status()
+        for i in range(gpu.n):
+            if ef:
+                for k in range(K):
+                    assert np.array_equal(_np(gpu.ef[k][i]), orc.ef[k][i]), f"E k={k} tensor {i} round {rnd}"
+            assert_close_1e6(_np(gpu.theta_g[i]), orc.theta_g[i], f"theta_g {i} round {rnd}")
+            assert_close_1e6(_np(gpu.outer_u[i]), orc.outer_u[i], f"u {i} round {rnd}")
+            for k in range(K):
+                assert np.array_equal(_np(gpu.theta_k[k][i]), _np(gpu.theta_g[i]))
+            orc.theta_g[i][...] = _np(gpu.theta_g[i]); orc.outer_u[i][...] = _np(gpu.outer_u[i])
+    gpu.close()
+
+
+def test_row_wise_rejects_rows_that_do_not_fit():
+    import dataclasses
+    from paper_2505_23725_b200 import binding
+    w = dataclasses.replace(_sync_workload(2, 8, [(2, 60000)]), quant_block=0)
+    gpu = gpu_for(w, [np.zeros((2, 60000), np.float32)])
+    with pytest.raises(binding.MulocoError) as e:
+        gpu.outer_sync(-1)
+    assert e.value.status == binding.ESHAPE
+    gpu.close()
