@@ -113,7 +113,7 @@ typedef struct {
                              may be NULL unless cfg.error_feedback is set                */
 } muloco_buffers;
 
-/* Algorithm 1, line 2.  Validates the arguments, records the tensor table,
+/* Algorithm 1, initialisation.  Validates the arguments, records the tensor table,
  * allocates the workspace (the only allocation the library makes), then
  * enqueues u <- 0, inner state <- 0 and theta_k <- theta_g for every worker.
  * `cuda_stream` is a cudaStream_t (NULL = the default stream).  n_tensors may
@@ -126,7 +126,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
 /* Releases workspace and tables (waits for the stream first). NULL is allowed. */
 MULOCO_API void muloco_destroy(muloco_ctx* ctx);
 
-/* Algorithm 1, lines 6-7 (Eq. 1) with the gradient given: one inner optimizer
+/* Algorithm 1, body of the inner loop (Eq. 1) with the gradient given: one inner optimizer
  * step for worker `worker` (0..K-1), or for all K workers batched when
  * worker == -1.  `grads` is a host table of device pointers: [n_tensors] for one
  * worker, [K][n_tensors] for all; each gradient has its tensor's shape and the
@@ -149,7 +149,7 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* ctx, int32_t worker, cons
 MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* ctx, int32_t worker,
                                      const void* const* host_grads, float lr_scale);
 
-/* Algorithm 1, lines 9-13 (Eqs. 2-3) for the tensors of fragment `fragment`
+/* Algorithm 1, outer step (Eqs. 2-3) for the tensors of fragment `fragment`
  * (0..J-1), or all tensors when fragment == -1, in one pass over memory:
  *     Psi = (1/K) sum_k (theta_g - theta_k)   (fp32, k ascending, then * 1/K)
  *     optional: Psi <- dequantise(quantise(Psi)) per block of quant_block elements

@@ -19,14 +19,14 @@ What each function follows:
   muon_step            Section 2 "Muon" (momentum, update with decoupled decay),
                        Section 5 "MuLoCo" (learning-rate rescale sqrt(n/m))
   adamw_step           Section 4.3 (first/second moments, decoupled decay)
-  pseudogradient       Eq. (2); Algorithm 1 lines 9 and 11
-  outer_nesterov       Eq. (3); Algorithm 1 lines 12-13
+  pseudogradient       Eq. (2); Algorithm 1 (parameter delta, all-reduce of the outer delta)
+  outer_nesterov       Eq. (3); Algorithm 1 (outer momentum, outer update)
   quantize_blocks      Section 2 "Compressed Communication" (linear quantisation)
                        in the per-block absmax form of the benchmark configs
   compressed_pseudogradient  Algorithm 2 (compression, error feedback) with the two
                        quantisations of Section 2 "Collectives for compressed communication"
   fragments_due        Section 2 "Partitioned Communication in Streaming DiLoCo"
-  MuLoCoOracle         Algorithm 1 (loop nest, initialisation line 2)
+  MuLoCoOracle         Algorithm 1 (loop nest and initialisation)
 
 Pins (tests/test_oracle_*.py, all run without a GPU): SVD closed form of the
 Newton-Schulz map, exact rational iterates of the scalar quintic, rank-1 Muon
@@ -335,7 +335,7 @@ class MuLoCoOracle:
         self.specs = list(specs)
         self.theta_g = [np.array(w, dtype=np.float32).reshape(s.rows, s.cols)
                         for w, s in zip(init, self.specs)]
-        # Algorithm 1 line 2: u <- 0, theta_i <- theta for all i
+        # Algorithm 1, initialisation: u <- 0, theta_i <- theta for all i
         self.outer_u = [np.zeros_like(w) for w in self.theta_g]
         self.theta_k = [[w.copy() for w in self.theta_g] for _ in range(cfg.K)]
         self.state1 = [[np.zeros_like(w) for w in self.theta_g] for _ in range(cfg.K)]
@@ -343,12 +343,12 @@ class MuLoCoOracle:
                         for w, s in zip(self.theta_g, self.specs)] for _ in range(cfg.K)]
         if cfg.error_feedback and (cfg.quant_stages != 2 or not cfg.quant_bits):
             raise ValueError("error feedback needs the two-stage quantised sync")
-        # Algorithm 2 line 4: E_i <- 0
+        # Algorithm 2, initialisation: E_i <- 0
         self.ef = [[np.zeros_like(w) for w in self.theta_g] for _ in range(cfg.K)] if cfg.error_feedback else None
         self.worker_step = [0] * cfg.K
         self.last_psi: Dict[int, np.ndarray] = {}
 
-    # Algorithm 1 lines 6-7 for one worker, gradients given
+    # Algorithm 1, inner loop body (Eq. 1) for one worker, gradients given
     def inner_step(self, worker: int, grads: Sequence[np.ndarray], lr_scale: float = 1.0):
         c = self.cfg
         self.worker_step[worker] += 1
@@ -372,7 +372,7 @@ class MuLoCoOracle:
         for k in range(self.cfg.K):
             self.inner_step(k, grads_k[k], lr_scale)
 
-    # Algorithm 1 lines 9-13 for the tensors of one fragment (-1: all), then
+    # Algorithm 1, outer step (Eqs. 2-3) for the tensors of one fragment (-1: all), then
     # the replicas of those tensors restart from the new global parameters.
     def outer_sync(self, fragment: int = -1):
         c = self.cfg

@@ -510,7 +510,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
 
   if (build_sync_tables(c) != MULOCO_OK) return bail(MULOCO_ECUDA);
 
-  // Algorithm 1, line 2: u <- 0, inner state <- 0, theta_k <- theta_g
+  // Algorithm 1, initialisation: u <- 0, inner state <- 0, theta_k <- theta_g
   for (int i = 0; i < n_tensors; ++i) {
     TensorInfo& t = c->T[i];
     const size_t bytes = (size_t)t.numel() * sizeof(float);

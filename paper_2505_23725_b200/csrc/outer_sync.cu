@@ -1,4 +1,4 @@
-// Outer synchronisation (Algorithm 1 lines 9-13, Eqs. 2-3) as ONE pass over memory:
+// Outer synchronisation (outer step of Algorithm 1, Eqs. 2-3) as ONE pass over memory:
 // pseudogradient over the K replicas, optional per-block quantise->dequantise,
 // Nesterov outer step, broadcast into the K replicas.  Pure HBM streaming:
 // (K+2) fp32 reads and (K+2) fp32 writes per parameter.
