@@ -183,6 +183,14 @@ def test_adamw_first_step_closed_form():
     assert np.allclose(th, want, rtol=2e-6, atol=1e-7)
     assert np.allclose(m, 0.1 * gd, rtol=1e-6)
     assert np.allclose(v, 0.01 * gd * gd, rtol=1e-6)
+    # where eps is felt: |g| = eps gives a half step, |g| << eps an almost vanishing one
+    # (eps is added to sqrt(v^), outside the root)
+    g2 = np.array([1e-8, -1e-8, 1e-10, 0.0], np.float32)
+    th = np.zeros(4, np.float32); m = np.zeros(4, np.float32); v = np.zeros(4, np.float32)
+    O.adamw_step(th, m, v, g2, t=1, lr=1.0, beta1=0.9, beta2=0.99, eps=1e-8, wd=0.0)
+    g2d = g2.astype(np.float64)
+    assert np.allclose(th, -(g2d / (np.abs(g2d) + 1e-8)), rtol=1e-5, atol=1e-12)
+    assert abs(th[0] + 0.5) < 1e-5 and abs(th[2]) < 0.0101
 
 
 def test_adamw_constant_gradient_and_no_bias_correction():
