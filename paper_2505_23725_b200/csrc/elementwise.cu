@@ -26,6 +26,10 @@ __device__ __forceinline__ float to_x<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ __nv_bfloat16 to_x<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+__device__ __forceinline__ void store_x2(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store_x2(__nv_bfloat16* p, float a, float b) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b);
+}
 __device__ __forceinline__ void store_x4(float* p, float4 u) { *reinterpret_cast<float4*>(p) = u; }
 __device__ __forceinline__ void store_x4(__nv_bfloat16* p, float4 u) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(u.x, u.y), hi = __floats2bfloat162_rn(u.z, u.w);
@@ -48,11 +52,21 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   const MatDesc d = mats[mat];
   // Tile order follows the tensor's own memory order, so that the CTAs resident at one
   // time read neighbouring addresses: tj fastest for a tensor stored s x l, ti fastest for
-  // one stored l x s (its rows are the j axis).
-  const int tiles_i = n_part / tiles_j;
-  const int ti = d.transposed ? (int)(blockIdx.x % tiles_i) : (int)(blockIdx.x / tiles_j);
-  const int tj = d.transposed ? (int)(blockIdx.x / tiles_i) : (int)(blockIdx.x % tiles_j);
-  const int64_t i0 = (int64_t)ti * PRO_TI, j0 = (int64_t)tj * PRO_TJ;
+  // one stored l x s (its rows are the j axis).  Tall tensors with an even s use 64 x 64 tiles
+  // (two consecutive i per lane); the grid has max(#32x128 tiles, #64x64 tiles) CTAs per matrix
+  // and the CTAs a tensor does not need write a zero partial sum.
+  const bool pair_ok = ((((uintptr_t)d.m) & 7) == 0) &&
+                       ((((uintptr_t)d.g) & ((src_mode == SRC_RAW_BF16 || (src_mode == SRC_MUON && g_is_bf16)) ? 3 : 7)) == 0);
+  const bool t64 = d.transposed && ((s & 1) == 0) && pair_ok;
+  const int tiles_i = t64 ? (int)((s + 63) / 64) : (int)((s + PRO_TI - 1) / PRO_TI);
+  const int tiles_jj = t64 ? (int)((l + 63) / 64) : tiles_j;
+  if ((int)blockIdx.x >= tiles_i * tiles_jj) {
+    if (threadIdx.x == 0) partials[(int64_t)mat * n_part + blockIdx.x] = 0.f;
+    return;
+  }
+  const int ti = d.transposed ? (int)(blockIdx.x % tiles_i) : (int)(blockIdx.x / tiles_jj);
+  const int tj = d.transposed ? (int)(blockIdx.x / tiles_i) : (int)(blockIdx.x % tiles_jj);
+  const int64_t i0 = (int64_t)ti * (t64 ? 64 : PRO_TI), j0 = (int64_t)tj * (t64 ? 64 : PRO_TJ);
   XT* Xm = X + (int64_t)mat * s * ldx;
   float ss = 0.f;
   const int tid = threadIdx.x;
@@ -72,9 +86,75 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
     return u;
   };
 
+  if (t64) {
+    // tensor is l x s: read rows j (64 consecutive i = 256 bytes per warp, two per lane), turn the
+    // tile through shared memory, write rows i of X (64 consecutive j per warp)
+    float (*t6)[65] = reinterpret_cast<float (*)[65]>(&tile[0][0]);
+    const int lane = tid & 31, w = tid >> 5;
+    const int64_t i = i0 + 2 * lane;
+    const bool src_bf16 = (src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16);
+    float2 gv[8], mv[8];
+    bool ok[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int64_t j = j0 + w + 8 * r;
+      ok[r] = (j < l) && (i < s);
+      gv[r] = make_float2(0.f, 0.f);
+      mv[r] = gv[r];
+      if (!ok[r]) continue;
+      const int64_t idx = j * s + i;
+      if (src_bf16) {
+        const uint32_t raw = __ldcs(reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(d.g) + idx));
+        gv[r] = make_float2(__uint_as_float(raw << 16), __uint_as_float(raw & 0xFFFF0000u));
+      } else {
+        gv[r] = __ldcs(reinterpret_cast<const float2*>(reinterpret_cast<const float*>(d.g) + idx));
+      }
+      if (src_mode == SRC_MUON) mv[r] = *reinterpret_cast<const float2*>(d.m + idx);
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int jj = w + 8 * r;
+      float2 u = make_float2(0.f, 0.f);
+      if (ok[r]) {
+        u = gv[r];
+        if (src_mode == SRC_MUON) {
+          float2 mn;
+          mn.x = fmaf(beta, mv[r].x, gv[r].x);
+          mn.y = fmaf(beta, mv[r].y, gv[r].y);
+          *reinterpret_cast<float2*>(d.m + (j0 + jj) * s + i) = mn;
+          if (nesterov) {
+            u.x = fmaf(beta, mn.x, gv[r].x);
+            u.y = fmaf(beta, mn.y, gv[r].y);
+          } else {
+            u = mn;
+          }
+        }
+        ss = fmaf(u.x, u.x, ss);
+        ss = fmaf(u.y, u.y, ss);
+      }
+      t6[jj][2 * lane] = u.x;
+      t6[jj][2 * lane + 1] = u.y;
+    }
+    __syncthreads();
+    const int64_t j = j0 + 2 * lane;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int ii = w + 8 * r;
+      const int64_t ix = i0 + ii;
+      if (ix >= s || j >= l) continue;
+      const float a0 = t6[2 * lane][ii], a1 = t6[2 * lane + 1][ii];
+      if (j + 1 < l) {
+        store_x2(Xm + ix * ldx + j, a0, a1);
+      } else {
+        Xm[ix * ldx + j] = to_x<XT>(a0);
+      }
+    }
+  }
   const bool vec4 = !d.transposed && ((l & 3) == 0) && ((ldx & 3) == 0) &&
                     ((((uintptr_t)d.g | (uintptr_t)d.m) & 15) == 0) && ((((uintptr_t)Xm) & 15) == 0);
-  if (vec4) {
+  if (t64) {
+    // handled above
+  } else if (vec4) {
     // tensor is s x l with 16-byte aligned rows: four consecutive j per thread.  All loads of
     // the thread's four rows are issued before the first store (the stores to m would
     // otherwise order the later loads behind them).
@@ -305,7 +385,9 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
 }  // namespace
 
 int prologue_partials_per_matrix(int64_t s, int64_t l) {
-  return (int)(((s + PRO_TI - 1) / PRO_TI) * ((l + PRO_TJ - 1) / PRO_TJ));
+  const int64_t a = ((s + PRO_TI - 1) / PRO_TI) * ((l + PRO_TJ - 1) / PRO_TJ);   // 32 x 128 tiles
+  const int64_t b = ((s + 63) / 64) * ((l + 63) / 64);                          // 64 x 64 tiles (tall tensors)
+  return (int)(a > b ? a : b);
 }
 
 void launch_prologue(cudaStream_t st, const MatDesc* mats, int n_mats, int64_t s, int64_t l,

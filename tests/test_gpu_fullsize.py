@@ -70,6 +70,9 @@ def _check_inner_and_sync(w, seed, slice_rows=64):
 
     opt.inner_step(-1, None, 1.0)                       # step 1: fills the momenta
     opt.sync_status()
+    # fresh gradients for the compared step, so that momentum and gradient point in different
+    # directions (with the same gradient twice, Nesterov's g + beta m is parallel to m)
+    synth.torch_fill_gradients(opt.grads, w.tensors, w.K, seed + 2, opt.device)
     before = {}
     for k, i in dict.fromkeys(pairs):
         t = w.tensors[i]
