@@ -114,7 +114,8 @@ typedef struct {
 } muloco_buffers;
 
 /* Algorithm 1, initialisation.  Validates the arguments, records the tensor table,
- * allocates the workspace (the only allocation the library makes), then
+ * allocates the library's own device memory (the Newton-Schulz workspace, small descriptor
+ * and pointer tables; the *_host calls add a gradient staging area on first use), then
  * enqueues u <- 0, inner state <- 0 and theta_k <- theta_g for every worker.
  * `cuda_stream` is a cudaStream_t (NULL = the default stream).  n_tensors may
  * be 0 for a context that only serves muloco_newton_schulz / muloco_quantize.
