@@ -5,8 +5,9 @@
 // One launch computes one of the three products of a Newton-Schulz iteration
 // (Section 2, "Muon": X_j = p(X X^T) X, p(x) = a x + b x^3 + c x^5) for every
 // matrix of a chunk; tiles of all matrices form one linear work list:
-//   GRAM  : A  = r^2 X X^T      symmetric: only tiles touching the upper triangle,
-//   POLY  : B  = b A + c A A    each 128-block stored directly and mirrored
+//   GRAM  : A  = r^2 X X^T      symmetric: only the tiles on or above the diagonal are computed
+//   POLY  : B  = b A + c A A    AND stored; a consumer fetches a block below the diagonal as the
+//                               transpose of its mirror image (an MN-major operand)
 //   APPLY : X' = r (a X + B X)
 //   FINAL : as APPLY, result goes to the parameter update / output sink
 // Operand forms: GRAM/POLY multiply a row-major matrix by its own transpose
@@ -49,8 +50,8 @@ constexpr int BK = 64;           // k slab per stage (64 bf16 = one 128-byte swi
 constexpr int UMMA_K = 16;
 constexpr int TC_THREADS = 192;
 // Pipeline depth is a template parameter: products that need all six staging blocks per epilogue
-// warp (POLY: addend + direct + mirrored; FINAL: addend + parameter ring) run 4 stages, those that
-// need four (GRAM: direct + mirrored; APPLY: addend + direct) run 5 in the same shared memory.
+// warp (FINAL: addend + parameter ring) run 4 stages, those that need at most four (GRAM: results;
+// POLY, APPLY: addend + results) run 5 in the same shared memory.
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;        // 16 KB: 128 rows x 64 k
 constexpr uint32_t B_STAGE_BYTES = 128 * BK * 2;       // 16 KB: this CTA's 128 columns of the right operand
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
@@ -71,6 +72,8 @@ struct TcParams {
   const float2* scales;
   const MatDesc* mats;
   int sink_mode;
+  int a_tri, b_tri;           // left / right operand is a symmetric matrix of which only the tiles on
+                              // or above the diagonal are stored
   int64_t s, l;
   int* status;
 };
@@ -281,12 +284,13 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
 //           MN-major 64 x 64 boxes)
 // tmC     : addend loads, 64 x 32 boxes (POLY: A, APPLY/FINAL: X)
 // tmD     : result stores, 64 x 32 boxes, 128-byte swizzle
-// tmT     : transposed result stores, 32 x 64 boxes, no swizzle (symmetric products)
+// tmS     : 64 x 64 boxes over the symmetric operand (POLY: A, APPLY/FINAL: B) for the k slabs
+//           whose block lies below the diagonal and is read from its mirror image
 template <int CG, bool B_MN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
-             const __grid_constant__ CUtensorMap tmT, const TcParams p) {
+             const __grid_constant__ CUtensorMap tmS, const TcParams p) {
   constexpr int BN = 128 * CG;                 // accumulator columns = tile columns
   constexpr int TM = 128 * CG;                 // tile rows (over the CTA pair)
   constexpr uint32_t TMEM_COLS = 2 * BN;
@@ -317,7 +321,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmT) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmS) : "memory");
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
@@ -356,31 +360,33 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const uint32_t full_local = smem_u32(&bar_full[stage]);
             const uint32_t sa = smem_base + stage * STAGE_BYTES;
             const uint32_t sb = sa + A_STAGE_BYTES;
-            if (CG == 1) {
-              mbar_expect_tx(full_local, cta_bytes);
-              tma_load_3d(sa, &tmA, full_local, kb * BK, a_row, mat);
-              if (!same) {
-                if (!B_MN) {
-                  tma_load_3d(sb, &tmB, full_local, kb * BK, b_off, mat);
-                } else {
-#pragma unroll
-                  for (int q = 0; q < 2; ++q)
-                    tma_load_3d(sb + q * (BK * 128), &tmB, full_local, b_off + q * 64, kb * BK, mat);
-                }
-              }
+            // blocks of a symmetric operand below the diagonal are not stored: their k slab is
+            // fetched from the mirror image as two 64 x 64 boxes (k rows, 64 operand rows each)
+            const int kT = (kb * BK) / TM;
+            const bool a_t = p.a_tri && kT < tt.x;
+            const bool b_t = p.b_tri && kT < tt.y;
+            const uint32_t bar = (CG == 1) ? full_local : map_to_rank(full_local, 0);
+            if (CG == 1) mbar_expect_tx(full_local, cta_bytes);
+            else if (rank == 0) mbar_expect_tx(full_local, 2u * cta_bytes);   // both CTAs' copies are counted here
+            auto load = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1) {
+              if (CG == 1) tma_load_3d(dst, map, bar, c0, c1, mat);
+              else tma_load_3d_pair(dst, map, bar, c0, c1, mat);
+            };
+            if (!a_t) {
+              load(sa, &tmA, kb * BK, a_row);
             } else {
-              // both CTAs' copies are counted on the barrier of rank 0, which expects the sum
-              const uint32_t full0 = map_to_rank(full_local, 0);
-              if (rank == 0) mbar_expect_tx(full_local, 2u * cta_bytes);
-              tma_load_3d_pair(sa, &tmA, full0, kb * BK, a_row, mat);
-              if (!same) {
-                if (!B_MN) {
-                  tma_load_3d_pair(sb, &tmB, full0, kb * BK, b_off, mat);
-                } else {
-#pragma unroll
-                  for (int q = 0; q < 2; ++q)
-                    tma_load_3d_pair(sb + q * (BK * 128), &tmB, full0, b_off + q * 64, kb * BK, mat);
-                }
+              load(sa, &tmS, a_row, kb * BK);
+              load(sa + BK * 128, &tmS, a_row + 64, kb * BK);
+            }
+            if (!same) {
+              if (B_MN) {
+                load(sb, &tmB, b_off, kb * BK);
+                load(sb + BK * 128, &tmB, b_off + 64, kb * BK);
+              } else if (!b_t) {
+                load(sb, &tmB, kb * BK, b_off);
+              } else {
+                load(sb, &tmS, b_off, kb * BK);
+                load(sb + BK * 128, &tmS, b_off + 64, kb * BK);
               }
             }
           }
@@ -393,8 +399,9 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
     if (rank == 0) {
-      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((B_MN ? 1u : 0u) << 16) |
-                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+      // fp32 accumulate, bf16 x bf16; bit 15 / bit 16: left / right operand is MN-major
+      constexpr uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) |
+                                  ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
       uint32_t stage = 0, phase = 0;
       int local_tile = 0;
       bool alive = true;
@@ -416,10 +423,15 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
               tc_fence_after();
               const uint32_t sa = smem_base + stage * STAGE_BYTES;
               const uint32_t sb = same ? sa : sa + A_STAGE_BYTES;
+              const int kT = (kb * BK) / TM;
+              const bool a_mn = p.a_tri && kT < tt.x;                 // as staged by the producer
+              const bool b_mn = B_MN || (p.b_tri && kT < tt.y);
+              const uint32_t idesc = idesc0 | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16);
 #pragma unroll
               for (int k = 0; k < BK / UMMA_K; ++k) {
-                const uint64_t adesc = make_sdesc(sa + k * (UMMA_K * 2), 16, 1024);
-                const uint64_t bdesc = B_MN ? make_sdesc(sb + k * (UMMA_K * 128), BK * 128, 1024)
+                const uint64_t adesc = a_mn ? make_sdesc(sa + k * (UMMA_K * 128), BK * 128, 1024)
+                                            : make_sdesc(sa + k * (UMMA_K * 2), 16, 1024);
+                const uint64_t bdesc = b_mn ? make_sdesc(sb + k * (UMMA_K * 128), BK * 128, 1024)
                                             : make_sdesc(sb + k * (UMMA_K * 2), 16, 1024);
                 tc_mma_bf16<CG>(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
               }
@@ -445,17 +457,16 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter+32)
     const int ew = warp - 2;               // staging slot of this warp
     const uint32_t epi = smem_base + STAGES * STAGE_BYTES + (uint32_t)ew * epi_warp_bytes(STAGES);
-    // staging blocks of this warp: addend 0/1, direct 0/1, mirrored 0/1
+    // staging blocks of this warp: addend 0/1 (when there is one), then results 0/1
     auto cin_buf = [&](uint32_t b) { return epi + b * EPI_BLOCK_BYTES; };
     const uint32_t o_first = (p.kind == GEMM_GRAM) ? 0u : 2u;     // the addend blocks come first when there are any
     auto out_buf = [&](uint32_t b) { return epi + (o_first + b) * EPI_BLOCK_BYTES; };
-    auto mir_buf = [&](uint32_t b) { return epi + (o_first + 2u + b) * EPI_BLOCK_BYTES; };
     const uint32_t cin_bar0 = smem_u32(&bar_cin[ew][0]);
     auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
     const bool has_cin = (p.kind != GEMM_GRAM);
     const bool stores = (p.kind != GEMM_FINAL);
     // parameter update through TMA: a ring of four 32 x 32 fp32 blocks in the staging space that
-    // the direct and mirrored results use in the other products
+    // after the addend blocks (the final product stages no results)
     auto w_buf = [&](uint32_t b) { return epi + (2u + b) * EPI_BLOCK_BYTES; };
     const uint32_t w_bar0 = smem_u32(&bar_w[ew][0]);
     auto w_bar = [&](uint32_t b) { return w_bar0 + b * 8u; };
@@ -479,7 +490,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int gj0 = TM * tt.y + c * 64;
-          if (gj0 < p.N && !(sym && (gj0 >> 7) < rb)) todo |= 1u << c;   // lower-triangle blocks come from their mirror image
+          if (gj0 < p.N) todo |= 1u << c;
         }
       }
       auto issue_cin = [&](int c) {
@@ -529,7 +540,6 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int c = __ffs(todo) - 1;
         todo &= todo - 1;
         const int gj0 = TM * tt.y + c * 64;
-        const bool mirror = sym && ((gj0 >> 7) > rb);
         if (has_cin) {
           if (todo) issue_cin(__ffs(todo) - 1);
           bool ok = mbar_wait(cin_bar(cin_used & 1u), (cin_used >> 1) & 1u, &abort_flag);
@@ -538,7 +548,6 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
         const uint32_t cbuf = cin_buf(cin_used & 1u);
         const uint32_t obuf = out_buf(st_count & 1u);
-        const uint32_t mbuf = mir_buf(st_count & 1u);
         if (stores) {
           if (lane == 0) bulk_wait_read_1();     // the block stored two steps ago has left this buffer
           __syncwarp();
@@ -682,19 +691,6 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
               u.w = pack_bf16x2(f[q * 8 + 6], f[q * 8 + 7]);
               sts128(obuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q) ^ (lane & 7)) << 4), u);
             }
-            if (mirror) {
-              // transposed block T[e][lane]: neighbouring lanes exchange one value so that
-              // each lane writes a packed pair of one transposed row
-              const bool odd = lane & 1;
-#pragma unroll
-              for (int e = 0; e < 32; e += 2) {
-                const float send = odd ? f[e] : f[e + 1];
-                const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
-                const uint32_t pk = odd ? pack_bf16x2(recv, f[e + 1]) : pack_bf16x2(f[e], recv);
-                const int trow = h * 32 + e + (odd ? 1 : 0);
-                sts32(mbuf + (uint32_t)trow * 64u + (uint32_t)((lane & ~1) * 2), pk);
-              }
-            }
           }
         }
         if (!alive) break;
@@ -704,7 +700,6 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           __syncwarp();
           if (lane == 0) {
             tma_store_3d(&tmD, obuf, gj0, gi0, mat);
-            if (mirror) tma_store_3d(&tmT, mbuf, gi0, gj0, mat);
             bulk_commit();
           }
           ++st_count;
@@ -855,9 +850,10 @@ struct TcGroupPlan {
   void* X[2];
   void* A;
   void* B;
-  // loads: K-major operand boxes, MN-major operand boxes; io: 64 x 32 boxes for addend loads and
-  // result stores; tr: 32 x 64 boxes for the transposed stores
-  CUtensorMap x_k[2], x_mn[2], x_io[2], a_k, a_io, a_tr, b_k, b_io, b_tr;
+  // k: K-major operand boxes (64 x 128); mn: MN-major operand boxes (64 x 64: X as the right
+  // operand of the apply, A and B for the blocks read from their mirror image); io: 64 x 32 boxes
+  // for addend loads and result stores
+  CUtensorMap x_k[2], x_mn[2], x_io[2], a_k, a_mn, a_io, b_k, b_mn, b_io;
   int2* tiles_sym = nullptr;
   int n_tiles_sym = 0;
   int2* tiles_full = nullptr;
@@ -889,10 +885,10 @@ TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1,
   }
   ok = ok && encode_map(&pl->a_k, A, s, s, chunk, lds, BK, 128, true);
   ok = ok && encode_map(&pl->a_io, A, s, s, chunk, lds, 64, 32, true);
-  ok = ok && encode_map(&pl->a_tr, A, s, s, chunk, lds, 32, 64, false);
+  ok = ok && encode_map(&pl->a_mn, A, s, s, chunk, lds, 64, BK, true);
   ok = ok && encode_map(&pl->b_k, B, s, s, chunk, lds, BK, 128, true);
   ok = ok && encode_map(&pl->b_io, B, s, s, chunk, lds, 64, 32, true);
-  ok = ok && encode_map(&pl->b_tr, B, s, s, chunk, lds, 32, 64, false);
+  ok = ok && encode_map(&pl->b_mn, B, s, s, chunk, lds, 64, BK, true);
   if (!ok) {
     snprintf(err, errlen, "cuTensorMapEncodeTiled failed for shape %lld x %lld", (long long)s, (long long)l);
     delete pl;
@@ -939,17 +935,19 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int kind, int n_mats, in
   Maps5 m;
   if (kind == GEMM_GRAM) {
     p.N = (int)pl->s; p.Kd = (int)pl->l; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
-    m = Maps5{&pl->x_k[xin], &pl->x_k[xin], &pl->a_io, &pl->a_io, &pl->a_tr};
+    m = Maps5{&pl->x_k[xin], &pl->x_k[xin], &pl->a_io, &pl->a_io, &pl->a_mn};
     return pl->cg == 2 ? launch_one<2, false, 5>(st, m, p, pl->n_sms) : launch_one<1, false, 5>(st, m, p, pl->n_sms);
   }
   if (kind == GEMM_POLY) {
     p.N = (int)pl->s; p.Kd = (int)pl->s; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
-    m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, &pl->b_tr};
-    return pl->cg == 2 ? launch_one<2, false, 4>(st, m, p, pl->n_sms) : launch_one<1, false, 4>(st, m, p, pl->n_sms);
+    p.a_tri = 1; p.b_tri = 1;
+    m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, &pl->a_mn};
+    return pl->cg == 2 ? launch_one<2, false, 5>(st, m, p, pl->n_sms) : launch_one<1, false, 5>(st, m, p, pl->n_sms);
   }
   p.N = (int)pl->l; p.Kd = (int)pl->s; p.tiles = pl->tiles_full; p.n_tiles_per_mat = pl->n_tiles_full;
   // FINAL stores nothing through tmD; the map still has to be a valid one
-  m = Maps5{&pl->b_k, &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin], &pl->x_io[1 - xin]};
+  p.a_tri = 1;      // the left operand is the polynomial B, stored on and above the diagonal
+  m = Maps5{&pl->b_k, &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin], &pl->b_mn};
   if (kind == GEMM_APPLY)
     return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
   return pl->cg == 2 ? launch_one<2, true, 4>(st, m, p, pl->n_sms) : launch_one<1, true, 4>(st, m, p, pl->n_sms);
