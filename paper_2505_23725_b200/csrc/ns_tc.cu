@@ -246,16 +246,6 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 // K-major operand  : rows of 64 bf16 (128 B) at 128 B pitch, 8-row groups 1024 B apart (SBO).
 // MN-major operand : 64-element (128 B) runs along MN, 8 k-rows per 1024 B group (SBO),
 //                    next 64-element MN atom `lbo` bytes further.
-__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
@@ -345,63 +335,77 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    uint32_t stage = 0, phase = 0;
-    bool alive = true;
-    for (int tile = unit; tile < total_tiles && alive; tile += n_units) {
-      const int mat = tile / p.n_tiles_per_mat;
-      const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
-      const bool same = sym && (tt.x == tt.y);     // diagonal tile: right slab == left slab
-      const int a_row = BM * (CG * tt.x + (int)rank);
-      const int b_off = TM * tt.y + 128 * (int)rank;
-      const uint32_t cta_bytes = A_STAGE_BYTES + (same ? 0u : B_STAGE_BYTES);
-      for (int kb = 0; kb < num_kb && alive; ++kb) {
-        if (lane == 0) {
-          if (mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, &abort_flag)) {
-            const uint32_t full_local = smem_u32(&bar_full[stage]);
-            const uint32_t sa = smem_base + stage * STAGE_BYTES;
-            const uint32_t sb = sa + A_STAGE_BYTES;
-            // blocks of a symmetric operand below the diagonal are not stored: their k slab is
-            // fetched from the mirror image as two 64 x 64 boxes (k rows, 64 operand rows each)
-            const int kT = (kb * BK) / TM;
-            const bool a_t = p.a_tri && kT < tt.x;
-            const bool b_t = p.b_tri && kT < tt.y;
-            const uint32_t bar = (CG == 1) ? full_local : map_to_rank(full_local, 0);
-            if (CG == 1) mbar_expect_tx(full_local, cta_bytes);
-            else if (rank == 0) mbar_expect_tx(full_local, 2u * cta_bytes);   // both CTAs' copies are counted here
-            auto load = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1) {
-              if (CG == 1) tma_load_3d(dst, map, bar, c0, c1, mat);
-              else tma_load_3d_pair(dst, map, bar, c0, c1, mat);
-            };
-            if (!a_t) {
-              load(sa, &tmA, kb * BK, a_row);
+    // One thread runs the whole loop; the other lanes wait at the end.
+    if (lane == 0) {
+      const uint32_t empty0 = smem_u32(&bar_empty[0]);
+      const uint32_t full0 = smem_u32(&bar_full[0]);
+      // both CTAs' copies are counted on the barrier of rank 0, which expects the sum
+      const uint32_t full0_bar = (CG == 2) ? map_to_rank(full0, 0) : full0;
+      uint32_t stage = 0, phase = 0;
+      bool alive = true;
+      for (int tile = unit; tile < total_tiles && alive; tile += n_units) {
+        const int mat = tile / p.n_tiles_per_mat;
+        const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
+        const bool same = sym && (tt.x == tt.y);     // diagonal tile: right slab == left slab
+        const int a_row = BM * (CG * tt.x + (int)rank);
+        const int b_off = TM * tt.y + 128 * (int)rank;
+        const uint32_t cta_bytes = A_STAGE_BYTES + (same ? 0u : B_STAGE_BYTES);
+        // blocks of a symmetric operand below the diagonal are not stored: their k slab is fetched
+        // from the mirror image as two 64 x 64 boxes (k rows, 64 operand rows each)
+        const int ka_mn = p.a_tri ? (TM / BK) * tt.x : 0;
+        const int kb_mn = p.b_tri ? (TM / BK) * tt.y : 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty0 + stage * 8u, phase ^ 1u, &abort_flag)) { alive = false; break; }
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_STAGE_BYTES;
+          const uint32_t bar = full0_bar + stage * 8u;
+          if (CG == 1) mbar_expect_tx(bar, cta_bytes);
+          else if (rank == 0) mbar_expect_tx(full0 + stage * 8u, 2u * cta_bytes);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1) {
+            if (CG == 1) tma_load_3d(dst, map, bar, c0, c1, mat);
+            else tma_load_3d_pair(dst, map, bar, c0, c1, mat);
+          };
+          const int k0 = kb * BK;
+          if (kb >= ka_mn) {
+            load(sa, &tmA, k0, a_row);
+          } else {
+            load(sa, &tmS, a_row, k0);
+            load(sa + BK * 128, &tmS, a_row + 64, k0);
+          }
+          if (!same) {
+            if (B_MN) {
+              load(sb, &tmB, b_off, k0);
+              load(sb + BK * 128, &tmB, b_off + 64, k0);
+            } else if (kb >= kb_mn) {
+              load(sb, &tmB, k0, b_off);
             } else {
-              load(sa, &tmS, a_row, kb * BK);
-              load(sa + BK * 128, &tmS, a_row + 64, kb * BK);
-            }
-            if (!same) {
-              if (B_MN) {
-                load(sb, &tmB, b_off, kb * BK);
-                load(sb + BK * 128, &tmB, b_off + 64, kb * BK);
-              } else if (!b_t) {
-                load(sb, &tmB, kb * BK, b_off);
-              } else {
-                load(sb, &tmS, b_off, kb * BK);
-                load(sb + BK * 128, &tmS, b_off + 64, kb * BK);
-              }
+              load(sb, &tmS, b_off, k0);
+              load(sb + BK * 128, &tmS, b_off + 64, k0);
             }
           }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        __syncwarp();
-        alive = (abort_flag == 0);
-        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
-    if (rank == 0) {
+    // One thread runs the whole loop (the other lanes wait at the end): per k slab it waits for the
+    // stage, issues four MMAs whose descriptors differ from the stage's base by a constant step,
+    // and commits the stage to both CTAs' empty barriers.
+    if (rank == 0 && lane == 0) {
       // fp32 accumulate, bf16 x bf16; bit 15 / bit 16: left / right operand is MN-major
       constexpr uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) |
                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+      // descriptor halves: high = SBO 1024 B | version 1 | 128-byte swizzle; low = address/16 | LBO/16 << 16
+      constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+      constexpr uint32_t LBO_K = (16u >> 4) << 16, LBO_MN = ((uint32_t)(BK * 128) >> 4) << 16;
+      constexpr uint32_t STEP_K = (UMMA_K * 2) >> 4, STEP_MN = (UMMA_K * 128) >> 4;
+      const uint32_t full0 = smem_u32(&bar_full[0]);
+      const uint32_t empty0 = smem_u32(&bar_empty[0]);
+      const uint32_t empty0_peer = (CG == 2) ? map_to_rank(empty0, 1) : 0u;
+      const uint32_t tfull0 = smem_u32(&bar_tfull[0]);
+      const uint32_t tfull0_peer = (CG == 2) ? map_to_rank(tfull0, 1) : 0u;
       uint32_t stage = 0, phase = 0;
       int local_tile = 0;
       bool alive = true;
@@ -409,49 +413,40 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int mat = tile / p.n_tiles_per_mat;
         const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
         const bool same = sym && (tt.x == tt.y);
-        const int acc = local_tile & 1;
+        // k slabs below these indices come from the mirror image (MN-major), as staged by the producer
+        const int ka_mn = p.a_tri ? (TM / BK) * tt.x : 0;
+        const int kb_mn = B_MN ? num_kb : (p.b_tri ? (TM / BK) * tt.y : 0);
+        const uint32_t acc = (uint32_t)local_tile & 1u;
         const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        if (lane == 0) {
-          if (mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, &abort_flag)) tc_fence_after();
-        }
-        __syncwarp();
-        alive = (abort_flag == 0);
-        for (int kb = 0; kb < num_kb && alive; ++kb) {
-          if (lane == 0) {
-            if (mbar_wait(smem_u32(&bar_full[stage]), phase, &abort_flag)) {
-              tc_fence_after();
-              const uint32_t sa = smem_base + stage * STAGE_BYTES;
-              const uint32_t sb = same ? sa : sa + A_STAGE_BYTES;
-              const int kT = (kb * BK) / TM;
-              const bool a_mn = p.a_tri && kT < tt.x;                 // as staged by the producer
-              const bool b_mn = B_MN || (p.b_tri && kT < tt.y);
-              const uint32_t idesc = idesc0 | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16);
+        const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
+        if (!mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, &abort_flag)) break;
+        tc_fence_after();
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full0 + stage * 8u, phase, &abort_flag)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = same ? sa : sa + A_STAGE_BYTES;
+          const bool a_mn = kb < ka_mn, b_mn = kb < kb_mn;
+          const uint32_t idesc = idesc0 | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16);
+          const uint32_t alo = (sa >> 4) | (a_mn ? LBO_MN : LBO_K), astep = a_mn ? STEP_MN : STEP_K;
+          const uint32_t blo = (sb >> 4) | (b_mn ? LBO_MN : LBO_K), bstep = b_mn ? STEP_MN : STEP_K;
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) {
-                const uint64_t adesc = a_mn ? make_sdesc(sa + k * (UMMA_K * 128), BK * 128, 1024)
-                                            : make_sdesc(sa + k * (UMMA_K * 2), 16, 1024);
-                const uint64_t bdesc = b_mn ? make_sdesc(sb + k * (UMMA_K * 128), BK * 128, 1024)
-                                            : make_sdesc(sb + k * (UMMA_K * 2), 16, 1024);
-                tc_mma_bf16<CG>(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-              }
-              const uint32_t e_local = smem_u32(&bar_empty[stage]);
-              tc_commit<CG>(e_local);
-              if (CG == 2) tc_commit<CG>(map_to_rank(e_local, 1));
-            }
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(alo + (uint32_t)k * astep);
+            const uint64_t bdesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(blo + (uint32_t)k * bstep);
+            tc_mma_bf16<CG>(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
           }
-          __syncwarp();
-          alive = (abort_flag == 0);
+          tc_commit<CG>(empty0 + stage * 8u);
+          if (CG == 2) tc_commit<CG>(empty0_peer + stage * 8u);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (alive && lane == 0) {
-          const uint32_t t_local = smem_u32(&bar_tfull[acc]);
-          tc_commit<CG>(t_local);
-          if (CG == 2) tc_commit<CG>(map_to_rank(t_local, 1));
+        if (alive) {
+          tc_commit<CG>(tfull0 + acc * 8u);
+          if (CG == 2) tc_commit<CG>(tfull0_peer + acc * 8u);
         }
-        __syncwarp();
       }
     }
+    __syncwarp();
   } else {
     // -------------------------------- epilogue --------------------------------
     const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter+32)
