@@ -142,8 +142,8 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* ctx, int32_t worker, cons
 
 /* As muloco_inner_step, but `host_grads` is a host table of HOST pointers
  * (pinned memory for full speed).  The gradients are copied to a device staging
- * area owned by the library (allocated on first use) by a copy stream of the
- * library's own, one section (group of same-shape matrices, then the AdamW tensors)
+ * area owned by the library (allocated on first use) by two copy streams of the
+ * library's own (alternating tensors), one section (group of same-shape matrices, then the AdamW tensors)
  * at a time; the step's kernels wait for their section only, so copies overlap the
  * compute of other sections and of the previous step.  The host buffers must stay
  * unchanged until the step has run (muloco_sync_status, or any wait on the stream). */

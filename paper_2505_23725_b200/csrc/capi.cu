@@ -117,8 +117,8 @@ struct muloco_ctx {
 
   // host-gradient staging: copies run on their own stream, one section (shape group, or the
   // AdamW tensors) at a time, so that the copy of a section overlaps the compute of the others
-  cudaStream_t copy_st = nullptr;
-  std::vector<cudaEvent_t> ev_copied, ev_consumed;   // per section
+  cudaStream_t copy_st = nullptr, copy_st2 = nullptr;   // two streams: per-copy overheads of one hide under the other
+  std::vector<cudaEvent_t> ev_copied, ev_copied2, ev_consumed;   // per section
   std::vector<char> consumed_valid;
   bool host_mode = false;                            // set while muloco_inner_step_host runs the step
   char* stage = nullptr;
@@ -542,9 +542,12 @@ MULOCO_API void muloco_destroy(muloco_ctx* c) {
   if (c->d_adam) cudaFree(c->d_adam);
   if (c->d_wmaps) cudaFree(c->d_wmaps);
   if (c->copy_st) cudaStreamSynchronize(c->copy_st);
+  if (c->copy_st2) cudaStreamSynchronize(c->copy_st2);
   for (cudaEvent_t e : c->ev_copied) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ev_copied2) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->ev_consumed) if (e) cudaEventDestroy(e);
   if (c->copy_st) cudaStreamDestroy(c->copy_st);
+  if (c->copy_st2) cudaStreamDestroy(c->copy_st2);
   if (c->stage) cudaFree(c->stage);
   for (FragTable& f : c->frags)
     if (f.d_segs) cudaFree(f.d_segs);
@@ -630,7 +633,10 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
   for (size_t gi = 0; gi < c->groups.size(); ++gi) {
     Group& g = c->groups[gi];
     const int count = (int)g.tensors.size() * nw;
-    if (c->host_mode) CK(cudaStreamWaitEvent(c->st, c->ev_copied[gi], 0));
+    if (c->host_mode) {
+      CK(cudaStreamWaitEvent(c->st, c->ev_copied[gi], 0));
+      CK(cudaStreamWaitEvent(c->st, c->ev_copied2[gi], 0));
+    }
     for (int m0 = 0; m0 < count; m0 += g.chunk) {
       const int cnt = std::min(g.chunk, count - m0);
       rs = run_ns_chunk(c, g, c->ws, c->d_mats + group_begin[gi] + m0, cnt, f.ns_mode, SRC_MUON,
@@ -644,7 +650,10 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
   }
   if (na) {
     const size_t sec = c->groups.size();
-    if (c->host_mode) CK(cudaStreamWaitEvent(c->st, c->ev_copied[sec], 0));
+    if (c->host_mode) {
+      CK(cudaStreamWaitEvent(c->st, c->ev_copied[sec], 0));
+      CK(cudaStreamWaitEvent(c->st, c->ev_copied2[sec], 0));
+    }
     {
       PhaseTimer t(c, MULOCO_PH_ADAMW);
       launch_adamw(c->st, c->d_adam, (int)na, units, g_is_bf16, f.adam_beta1, f.adam_beta2, f.adam_eps);
@@ -688,11 +697,14 @@ MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* c, int32_t worker, c
   const size_t n_sec = c->groups.size() + 1;           // shape groups, then the AdamW tensors
   if (!c->copy_st) {
     CK(cudaStreamCreateWithFlags(&c->copy_st, cudaStreamNonBlocking));
+    CK(cudaStreamCreateWithFlags(&c->copy_st2, cudaStreamNonBlocking));
     c->ev_copied.assign(n_sec, nullptr);
+    c->ev_copied2.assign(n_sec, nullptr);
     c->ev_consumed.assign(n_sec, nullptr);
     c->consumed_valid.assign(n_sec, 0);
     for (size_t s2 = 0; s2 < n_sec; ++s2) {
       CK(cudaEventCreateWithFlags(&c->ev_copied[s2], cudaEventDisableTiming));
+      CK(cudaEventCreateWithFlags(&c->ev_copied2[s2], cudaEventDisableTiming));
       CK(cudaEventCreateWithFlags(&c->ev_consumed[s2], cudaEventDisableTiming));
     }
   }
@@ -701,18 +713,24 @@ MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* c, int32_t worker, c
   // belong to different pinned allocations, which a single copy must not span), signal.
   for (size_t sec = 0; sec < n_sec; ++sec) {
     const std::vector<int>& ids = sec < c->groups.size() ? c->groups[sec].tensors : c->adam_ids;
-    if (c->consumed_valid[sec]) CK(cudaStreamWaitEvent(c->copy_st, c->ev_consumed[sec], 0));
+    if (c->consumed_valid[sec]) {
+      CK(cudaStreamWaitEvent(c->copy_st, c->ev_consumed[sec], 0));
+      CK(cudaStreamWaitEvent(c->copy_st2, c->ev_consumed[sec], 0));
+    }
     {
       PhaseTimer t(c, MULOCO_PH_COPY, c->copy_st);
+      int which = 0;
       for (int k = k0; k < k1; ++k)
         for (int i : ids) {
           const void* src = host_grads[(size_t)(k - k0) * n + i];
           char* dst = c->stage + c->stage_off[(size_t)k * n + i];
           dev[(size_t)(k - k0) * n + i] = dst;
-          CK(cudaMemcpyAsync(dst, src, (size_t)c->T[i].numel() * elt, cudaMemcpyHostToDevice, c->copy_st));
+          CK(cudaMemcpyAsync(dst, src, (size_t)c->T[i].numel() * elt, cudaMemcpyHostToDevice,
+                             (which++ & 1) ? c->copy_st2 : c->copy_st));
         }
     }
     CK(cudaEventRecord(c->ev_copied[sec], c->copy_st));
+    CK(cudaEventRecord(c->ev_copied2[sec], c->copy_st2));
   }
   c->host_mode = true;
   const muloco_status rs = muloco_inner_step(c, worker, dev.data(), lr_scale);
