@@ -142,15 +142,18 @@ def time_oracle_sample(w, seed=0):
 
     rng = np.random.default_rng(seed)
     layer = [t for t in w.tensors if t.kind == configs.MUON and t.name.startswith("l0.")]
-    pm = sum(t.numel for t in layer)
-    Ws = [(0.02 * rng.standard_normal((t.rows, t.cols))).astype(np.float32) for t in layer]
-    Ms = [np.zeros_like(x) for x in Ws]
-    Gs = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) for t in layer]
-    t0 = time.perf_counter()
-    for W, M, G in zip(Ws, Ms, Gs):
-        O.muon_step(W, M, G, lr=w.muon_lr, beta=w.muon_beta, wd=w.muon_wd, nesterov=w.muon_nesterov)
-    t_muon = time.perf_counter() - t0
-    pa = 1 << 20
+    reps_muon = 4 if layer and max(max(t.rows, t.cols) for t in layer) <= 4096 else 1   # (layer, worker) pairs sampled
+    pm = sum(t.numel for t in layer) * reps_muon
+    t_muon = 0.0
+    for _ in range(reps_muon):
+        Ws = [(0.02 * rng.standard_normal((t.rows, t.cols))).astype(np.float32) for t in layer]
+        Ms = [np.zeros_like(x) for x in Ws]
+        Gs = [rng.standard_normal((t.rows, t.cols)).astype(np.float32) for t in layer]
+        t0 = time.perf_counter()
+        for W, M, G in zip(Ws, Ms, Gs):
+            O.muon_step(W, M, G, lr=w.muon_lr, beta=w.muon_beta, wd=w.muon_wd, nesterov=w.muon_nesterov)
+        t_muon += time.perf_counter() - t0
+    pa = 1 << 22
     th = rng.standard_normal(pa).astype(np.float32); m = np.zeros_like(th); v = np.zeros_like(th)
     g = rng.standard_normal(pa).astype(np.float32)
     t0 = time.perf_counter()
@@ -175,8 +178,8 @@ def time_oracle_sample(w, seed=0):
     n_adam = w.n_params - n_muon
     t_round = w.H * w.K * (n_muon / pm * t_muon + n_adam / pa * t_adam) + w.n_params / ps * t_sync
     value = w.K * w.n_params * w.H / t_round
-    sample = (f"one layer x one worker Muon step ({len(layer)} matrices, {pm} params, {t_muon:.2f} s), "
-              f"AdamW on 2^20 elements ({t_adam:.3f} s), outer sync of {ps} params x K={w.K} replicas "
+    sample = (f"{reps_muon} (layer, worker) Muon steps ({reps_muon * len(layer)} matrices, {pm} params, {t_muon:.2f} s), "
+              f"AdamW on 2^22 elements ({t_adam:.3f} s), outer sync of {ps} params x K={w.K} replicas "
               f"({t_sync:.2f} s); extrapolated linearly to a full round of H={w.H} steps")
     return value, sample, t_muon + t_adam + t_sync
 
