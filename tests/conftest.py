@@ -12,6 +12,16 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
 
+def pytest_sessionstart(session):
+    """Build libmuloco.so when it is missing or older than its sources (a build step, not a
+    fallback: without nvcc the tests that need the library fail with the binding's own message)."""
+    try:
+        from paper_2505_23725_b200 import build
+        build.build_library(force=False)
+    except Exception as e:                      # noqa: BLE001 - report and let the tests speak
+        sys.stderr.write(f"libmuloco.so was not (re)built: {e}\n")
+
+
 def _cuda_ok():
     try:
         import torch
