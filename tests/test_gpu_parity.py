@@ -59,7 +59,10 @@ def test_cfg0_full_round_fp32_mode():
 # Newton-Schulz on its own
 # ---------------------------------------------------------------------------
 NS_SHAPES = [(1, 128, 128), (2, 128, 352), (2, 352, 128), (1, 256, 512), (3, 768, 768), (1, 200, 300),
-             (2, 100, 72), (1, 64, 64), (1, 8, 24), (2, 1024, 2816), (1, 2816, 1024), (5, 384, 640)]
+             (2, 100, 72), (1, 64, 64), (1, 8, 24), (2, 1024, 2816), (1, 2816, 1024), (5, 384, 640),
+             # ragged against every tile size: rows/cols off the 64-, 128- and 256-grids, odd pitches
+             (2, 257, 513), (1, 130, 1000), (3, 511, 129), (1, 96, 1031), (1, 1000, 1000), (2, 640, 641),
+             (40, 512, 512), (150, 256, 256)]
 
 
 @pytest.fixture(scope="module")
