@@ -48,7 +48,8 @@ typedef enum {
   MULOCO_ESHAPE = 2,     /* unsupported shape */
   MULOCO_ENOMEM = 3,     /* workspace allocation failed */
   MULOCO_ECUDA = 4,      /* CUDA runtime/driver error, or no device */
-  MULOCO_ENONFINITE = 5, /* device saw a non-finite pseudogradient */
+  MULOCO_ENONFINITE = 5, /* device saw a non-finite pseudogradient, or a non-finite gradient /
+                            momentum of a hidden matrix (its Frobenius norm)          */
   MULOCO_ETIMEOUT = 6,   /* a bounded wait inside a kernel ran out */
   MULOCO_ESTATE = 7      /* call order / state blob mismatch */
 } muloco_status;

@@ -242,7 +242,7 @@ muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_m
     PhaseTimer t(c, MULOCO_PH_PROLOGUE);
     launch_prologue(c->st, d_mats, n_mats, g.s, g.l, src_mode, g_is_bf16, f.muon_beta, f.muon_nesterov,
                     X[0], mode == MULOCO_NS_FP32, g.ldx, partials);
-    launch_finalize_scales(c->st, partials, g.n_part, n_mats, f.ns_eps, scales);
+    launch_finalize_scales(c->st, partials, g.n_part, n_mats, f.ns_eps, scales, c->d_status);
     c->launches += 2;
   }
   PhaseTimer t(c, MULOCO_PH_NS);
@@ -947,7 +947,8 @@ MULOCO_API muloco_status muloco_sync_status(muloco_ctx* c) {
   if (h) CK(cudaMemset(c->d_status, 0, sizeof(int)));
   if (h & ST_TIMEOUT) return fail(c, MULOCO_ETIMEOUT, "a bounded wait inside a kernel ran out");
   if (h & ST_BOUNDS) return fail(c, MULOCO_ECUDA, "a kernel rejected an out-of-range index");
-  if (h & ST_NONFINITE) return fail(c, MULOCO_ENONFINITE, "non-finite pseudogradient");
+  if (h & ST_NONFINITE)
+    return fail(c, MULOCO_ENONFINITE, "non-finite value: a pseudogradient, or the Newton-Schulz input of a hidden matrix");
   return MULOCO_OK;
 }
 

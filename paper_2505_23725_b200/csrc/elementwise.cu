@@ -288,7 +288,7 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
 }
 
 __global__ void finalize_scales_kernel(const float* __restrict__ partials, int n_part, int n_mats,
-                                       float eps, float2* __restrict__ scales) {
+                                       float eps, float2* __restrict__ scales, int* __restrict__ status) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= n_mats) return;
@@ -300,6 +300,8 @@ __global__ void finalize_scales_kernel(const float* __restrict__ partials, int n
   if (lane == 0) {
     const double r = 1.0 / (sqrt(acc) + (double)eps);
     scales[warp] = make_float2((float)(r * r), (float)r);
+    // a NaN or infinity anywhere in the input (gradient or momentum) shows up here
+    if (status && !(acc <= 1.0e300)) atomicOr(status, ST_NONFINITE);
   }
 }
 
@@ -413,11 +415,11 @@ void launch_prologue(cudaStream_t st, const MatDesc* mats, int n_mats, int64_t s
 }
 
 void launch_finalize_scales(cudaStream_t st, const float* partials, int n_part, int n_mats, float eps,
-                            float2* scales) {
+                            float2* scales, int* status) {
   if (n_mats <= 0) return;
   const int threads = 128;
   const int blocks = (n_mats * 32 + threads - 1) / threads;
-  finalize_scales_kernel<<<blocks, threads, 0, st>>>(partials, n_part, n_mats, eps, scales);
+  finalize_scales_kernel<<<blocks, threads, 0, st>>>(partials, n_part, n_mats, eps, scales, status);
 }
 
 void launch_adamw(cudaStream_t st, const AdamSeg* segs, int n_segs, int64_t n_units, int g_is_bf16,

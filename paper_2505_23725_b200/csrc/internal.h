@@ -39,7 +39,7 @@ void launch_prologue(cudaStream_t st, const MatDesc* mats, int n_mats, int64_t s
 int prologue_partials_per_matrix(int64_t s, int64_t l);
 // scales[slot] = { r*r, r } with r = 1 / (sqrt(sum partials) + eps)
 void launch_finalize_scales(cudaStream_t st, const float* partials, int n_part, int n_mats,
-                            float eps, float2* scales);
+                            float eps, float2* scales, int* status = nullptr);
 
 // fp32 Newton-Schulz engine (CUDA cores).  One call = one of the three products
 // of an iteration for all matrices of a chunk.

@@ -549,3 +549,22 @@ def test_row_wise_rejects_rows_that_do_not_fit():
         gpu.outer_sync(-1)
     assert e.value.status == binding.ESHAPE
     gpu.close()
+
+
+def test_nonfinite_gradient_of_a_hidden_matrix_is_reported():
+    import torch
+    from paper_2505_23725_b200 import binding
+    w = configs.mini_workload(K=1, H=1, L=1, d=64, F=96, ns_mode="bf16")
+    rng = np.random.default_rng(8)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    gs = synth.host_gradients(rng, w.tensors)
+    gpu.inner_step(-1, to_dev([gs]))
+    gpu.sync_status()                                   # finite gradients: no complaint
+    gs[2][3, 5] = np.nan
+    gpu.inner_step(-1, to_dev([gs]))
+    with pytest.raises(binding.MulocoError) as e:
+        gpu.sync_status()
+    assert e.value.status == binding.ENONFINITE
+    gpu.sync_status()                                   # the flag is cleared once read
+    gpu.close()
