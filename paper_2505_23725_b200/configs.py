@@ -142,6 +142,24 @@ def diloco_baseline(w: Workload) -> Workload:
     return dataclasses.replace(w, tensors=ts, name=w.name + "-diloco")
 
 
+def cosine_lr_scale(step: int, total_steps: int, warmup_steps: int = 0,
+                    final_fraction: float = 0.1) -> float:
+    """The learning-rate multiplier for inner step `step` (0-based) of `total_steps`: a linear
+    warm-up over `warmup_steps`, then a half cosine from 1 down to `final_fraction` of the peak
+    (Section 5: cosine decay to 0.1x the maximum).  The result is the `lr_scale` argument of the
+    inner step; the library itself holds no schedule."""
+    import math
+    if total_steps <= 0 or not 0 <= step:
+        raise ValueError("need total_steps > 0 and step >= 0")
+    if not 0 <= warmup_steps < total_steps:
+        raise ValueError("warmup_steps must lie in [0, total_steps)")
+    if step < warmup_steps:
+        return (step + 1) / warmup_steps
+    span = max(1, total_steps - 1 - warmup_steps)
+    t = min(1.0, (step - warmup_steps) / span)
+    return final_fraction + (1.0 - final_fraction) * 0.5 * (1.0 + math.cos(math.pi * t))
+
+
 def mini_workload(K=2, H=2, J=1, quant_bits=0, ns_mode="fp32", L=2, d=128, F=352,
                   vocab=0, norms=False, **kw) -> Workload:
     """A small custom workload for tests."""

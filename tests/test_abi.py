@@ -83,3 +83,20 @@ def test_product_does_not_import_the_oracle():
         if f.endswith(".py"):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2505_23725_b200" not in text and "ctypes" not in text
+
+
+def test_cosine_schedule_endpoints_midpoint_and_monotonicity():
+    """Section 5: cosine decay to 0.1x the maximum.  Closed-form points of the half cosine."""
+    from paper_2505_23725_b200.configs import cosine_lr_scale as f
+    T, W = 1001, 100
+    assert f(0, T) == 1.0 and abs(f(T - 1, T) - 0.1) < 1e-15
+    assert abs(f(500, T) - 0.55) < 1e-12                      # midpoint: (1 + 0.1) / 2
+    assert abs(f(250, T) - (0.1 + 0.9 * 0.5 * (1 + 2 ** -0.5))) < 1e-12   # quarter: cos(pi/4)
+    assert f(0, T, W) == 1 / W and f(W - 1, T, W) == 1.0 and f(W, T, W) == 1.0
+    xs = [f(t, T, W) for t in range(W, T)]
+    assert all(a >= b for a, b in zip(xs, xs[1:])) and abs(xs[-1] - 0.1) < 1e-15
+    assert f(5 * T, T) == pytest.approx(0.1)                  # past the end: stays at the floor
+    with pytest.raises(ValueError):
+        f(0, 0)
+    with pytest.raises(ValueError):
+        f(0, 10, 10)
