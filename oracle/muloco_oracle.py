@@ -7,9 +7,9 @@ imports nothing from the product (no shared kernels, tables or helpers).
 
 Arithmetic: every state array is stored as float32 (as on the GPU).  Each
 operation loads to float64, computes, and rounds ONCE to float32 on store.
-The only exception is the block quantiser (and the pseudogradient that feeds
-it), which is written in exact float32 operations so that integer codes are
-reproducible bit for bit.
+The only exception is the compressors (block quantiser, top-k) and the
+pseudogradient that feeds them, which are written in exact float32 operations
+so that integer codes and kept sets are reproducible bit for bit.
 
 Hyper-parameters cross the library boundary as float32; callers that want to
 mirror the library pass values that are already float32-representable.
@@ -25,6 +25,9 @@ What each function follows:
                        in the per-block absmax form of the benchmark configs
   compressed_pseudogradient  Algorithm 2 (compression, error feedback) with the two
                        quantisations of Section 2 "Collectives for compressed communication"
+  topk_sparsify        Section 2 "Compressed Communication" (top-k sparsification)
+  sparsified_pseudogradient  Algorithm 2 with top-k as the compressor, sparsified once before
+                       the all-gather (Appendix, "Assumptions around the collective used")
   fragments_due        Section 2 "Partitioned Communication in Streaming DiLoCo"
   MuLoCoOracle         Algorithm 1 (loop nest and initialisation)
 
@@ -33,7 +36,8 @@ Newton-Schulz map, exact rational iterates of the scalar quintic, rank-1 Muon
 step, K=1 equivalence with plain Muon, identical-gradient pseudogradient,
 Proposition 4.2's nuclear-norm identity, AdamW / outer-step closed forms,
 quantiser error bound / ties / idempotence, streaming coverage, two-stage
-compression (K=1 collapse, error bound, error-feedback conservation).
+compression (K=1 collapse, error bound, error-feedback conservation), top-k
+(brute-force selection, best k-term approximation by enumeration, ties, counts).
 Parity unpinned: none of the functions above; the bf16 production mode of the
 GPU Newton-Schulz has no pin other than this oracle (tolerance 2e-2).
 """
@@ -230,6 +234,59 @@ def compressed_pseudogradient(theta_g, thetas: Sequence[np.ndarray], bits: int, 
     return psi.reshape(tg.shape)
 
 
+def topk_count(n: int, fraction: float) -> int:
+    """How many entries of a tensor of n elements top-k keeps: floor(fraction * n), in double
+    precision with `fraction` first rounded to float32 (how it crosses the library boundary),
+    at least 1 and at most n."""
+    return int(min(n, max(1, math.floor(float(np.float32(fraction)) * n))))
+
+
+def topk_sparsify(x, fraction: float):
+    """Top-k sparsification of one weight matrix (Section 2, "Compressed Communication"): the
+    k% entries of largest magnitude are kept, every other entry becomes 0.
+
+    The selection is over the whole tensor.  With kk = topk_count(n, fraction) and tau the
+    kk-th largest magnitude, the entries with |x| >= tau are kept: entries tied with the
+    kk-th one are all kept, so the result does not depend on an order among equals.
+    Returns a float32 array of x's shape."""
+    a = np.asarray(x, dtype=np.float32)
+    flat = np.abs(a).reshape(-1)
+    n = flat.size
+    if n == 0:
+        return a.copy()
+    kk = topk_count(n, fraction)
+    tau = np.sort(flat)[n - kk]
+    return np.where(np.abs(a) >= tau, a, np.float32(0)).astype(np.float32)
+
+
+def sparsified_pseudogradient(theta_g, thetas: Sequence[np.ndarray], fraction: float,
+                              ef: Optional[Sequence[np.ndarray]] = None, ef_beta: float = 1.0):
+    """Algorithm 2 with top-k as the compressor; the sparsified deltas are gathered from all
+    workers, so each is sparsified once and nothing is compressed after the mean (Appendix,
+    "Assumptions around the collective used").  In float32, workers in ascending order:
+
+      per worker i:  Delta_i = theta - theta_i
+                     with EF:  E_i <- beta E_i + Delta_i;  Delta~_i = topk(E_i);  E_i <- E_i - Delta~_i
+                     else:     Delta~_i = topk(Delta_i)
+      Psi = (1/K) sum_i Delta~_i
+
+    `ef` (float32 arrays, one per worker) is updated in place.  Returns Psi (float32)."""
+    tg = np.asarray(theta_g, dtype=np.float32)
+    K = len(thetas)
+    acc = np.zeros_like(tg)
+    beta = np.float32(ef_beta)
+    for i, th in enumerate(thetas):
+        delta = (tg - np.asarray(th, dtype=np.float32)).astype(np.float32)
+        if ef is not None:
+            e = ((beta * ef[i]).astype(np.float32) + delta).astype(np.float32)
+            c = topk_sparsify(e, fraction)
+            ef[i][...] = (e - c).astype(np.float32)
+        else:
+            c = topk_sparsify(delta, fraction)
+        acc = (acc + c).astype(np.float32)
+    return (acc * np.float32(1.0 / K)).astype(np.float32)
+
+
 def pack_int4(codes):
     """Two 4-bit two's-complement codes per byte along a row, element 2j in the
     low nibble; a row with an odd number of elements pads the last high nibble
@@ -305,8 +362,9 @@ class OracleConfig:
     quant_block: int = 128        # 0 = one block per row (row-wise quantisation)
     quant_stages: int = 1         # 1: quantise the averaged pseudogradient once (benchmark form);
                                   # 2: per-worker quantisation, high-precision mean, second quantisation
-    error_feedback: bool = False  # Algorithm 2 (needs quant_stages = 2)
+    error_feedback: bool = False  # Algorithm 2 (needs quant_stages = 2 or topk_fraction > 0)
     ef_beta: float = 1.0
+    topk_fraction: float = 0.0    # > 0: top-k sparsification of every worker's delta (no quantiser)
 
     def f32(self) -> "OracleConfig":
         """The same configuration with every real hyper-parameter rounded to
@@ -314,7 +372,7 @@ class OracleConfig:
         r = lambda x: float(np.float32(x))
         d = dict(self.__dict__)
         for k in ("muon_lr", "muon_beta", "muon_wd", "ns_eps", "adam_lr", "adam_beta1",
-                  "adam_beta2", "adam_eps", "adam_wd", "outer_lr", "outer_momentum", "ef_beta"):
+                  "adam_beta2", "adam_eps", "adam_wd", "outer_lr", "outer_momentum", "ef_beta", "topk_fraction"):
             d[k] = r(d[k])
         d["ns_coeffs"] = tuple(r(x) for x in self.ns_coeffs)
         return OracleConfig(**d)
@@ -341,8 +399,12 @@ class MuLoCoOracle:
         self.state1 = [[np.zeros_like(w) for w in self.theta_g] for _ in range(cfg.K)]
         self.state2 = [[np.zeros_like(w) if s.kind == "adamw" else None
                         for w, s in zip(self.theta_g, self.specs)] for _ in range(cfg.K)]
-        if cfg.error_feedback and (cfg.quant_stages != 2 or not cfg.quant_bits):
-            raise ValueError("error feedback needs the two-stage quantised sync")
+        if cfg.topk_fraction and cfg.quant_bits:
+            raise ValueError("top-k sparsification and quantisation are not combined")
+        if not 0.0 <= cfg.topk_fraction <= 1.0:
+            raise ValueError("topk_fraction must lie in [0, 1]")
+        if cfg.error_feedback and not cfg.topk_fraction and (cfg.quant_stages != 2 or not cfg.quant_bits):
+            raise ValueError("error feedback needs the two-stage quantised sync or top-k")
         # Algorithm 2, initialisation: E_i <- 0
         self.ef = [[np.zeros_like(w) for w in self.theta_g] for _ in range(cfg.K)] if cfg.error_feedback else None
         self.worker_step = [0] * cfg.K
@@ -381,7 +443,10 @@ class MuLoCoOracle:
                 continue
             reps = [self.theta_k[k][i] for k in range(c.K)]
             blk = c.quant_block if c.quant_block > 0 else s.cols
-            if c.quant_bits and c.quant_stages == 2:
+            if c.topk_fraction:
+                efs = [self.ef[k][i] for k in range(c.K)] if self.ef is not None else None
+                psi = sparsified_pseudogradient(self.theta_g[i], reps, c.topk_fraction, efs, c.ef_beta)
+            elif c.quant_bits and c.quant_stages == 2:
                 efs = [self.ef[k][i] for k in range(c.K)] if self.ef is not None else None
                 psi = compressed_pseudogradient(self.theta_g[i], reps, c.quant_bits, blk, efs, c.ef_beta)
             elif c.quant_bits:

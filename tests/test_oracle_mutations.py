@@ -66,6 +66,24 @@ MUTATIONS = [
      "ef[i][...] = e", ["test_error_feedback_conserves_what_was_not_sent"]),
     ("error feedback: delta not added", "e = ((beta * ef[i]).astype(np.float32) + delta).astype(np.float32)",
      "e = (beta * ef[i]).astype(np.float32) + np.float32(0) * delta", ["test_error_feedback_conserves_what_was_not_sent"]),
+    ("top-k: smallest magnitudes kept", "tau = np.sort(flat)[n - kk]\n    return np.where(np.abs(a) >= tau, a, np.float32(0)).astype(np.float32)",
+     "tau = np.sort(flat)[kk - 1]\n    return np.where(np.abs(a) <= tau, a, np.float32(0)).astype(np.float32)",
+     ["test_topk_matches_brute_force_selection"]),
+    ("top-k: selection on signed values", "tau = np.sort(flat)[n - kk]\n    return np.where(np.abs(a) >= tau, a,",
+     "tau = np.sort(a.reshape(-1))[n - kk]\n    return np.where(a >= tau, a,", ["test_topk_matches_brute_force_selection"]),
+    ("top-k: one entry too many", "tau = np.sort(flat)[n - kk]", "tau = np.sort(flat)[max(n - kk - 1, 0)]",
+     ["test_topk_matches_brute_force_selection", "test_topk_is_the_best_k_term_approximation"]),
+    ("top-k: selection per row", "    flat = np.abs(a).reshape(-1)\n    n = flat.size\n    if n == 0:\n        return a.copy()\n",
+     "    if a.ndim == 2 and a.shape[0] > 1:\n        return np.stack([topk_sparsify(r, fraction) for r in a])\n"
+     "    flat = np.abs(a).reshape(-1)\n    n = flat.size\n    if n == 0:\n        return a.copy()\n",
+     ["test_topk_ties_counts_and_degenerate_inputs", "test_topk_matches_brute_force_selection"]),
+    ("top-k: count rounded up", "max(1, math.floor(float(np.float32(fraction)) * n))", "max(1, math.ceil(float(np.float32(fraction)) * n))",
+     ["test_topk_ties_counts_and_degenerate_inputs", "test_topk_matches_brute_force_selection"]),
+    ("top-k: mean sparsified instead of the workers' deltas", "            c = topk_sparsify(delta, fraction)\n        acc = (acc + c).astype(np.float32)\n    return (acc * np.float32(1.0 / K)).astype(np.float32)",
+     "            c = delta\n        acc = (acc + c).astype(np.float32)\n    return topk_sparsify((acc * np.float32(1.0 / K)).astype(np.float32), fraction)",
+     ["test_sparsified_pseudogradient_definitions_and_error_feedback"]),
+    ("top-k error feedback: sent part left in the accumulator", "ef[i][...] = (e - c).astype(np.float32)", "ef[i][...] = e",
+     ["test_sparsified_pseudogradient_definitions_and_error_feedback"]),
     ("sync: replicas not reset", "self.theta_k[k][i][...] = self.theta_g[i]", "pass",
      ["test_j1_equals_non_streaming_and_state_is_kept_across_syncs", "test_streaming_touches_each_fragment_once_per_period",
       "test_k1_outer_identity_reproduces_plain_muon"]),

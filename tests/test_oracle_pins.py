@@ -421,3 +421,120 @@ def test_row_wise_quantisation_is_one_block_per_row():
     assert scales.shape == (4, 1)
     assert np.array_equal(scales[:, 0], (np.abs(x).max(axis=1) / np.float32(127)).astype(np.float32))
     assert np.all(np.abs(codes).max(axis=1) == 127)
+
+
+# ---- top-k sparsification (Section 2, "Compressed Communication") ------------
+def _topk_brute(x, kk):
+    """Plain selection: walk the entries from the largest magnitude down, keep the first kk and
+    everything tied with the kk-th."""
+    flat = [float(v) for v in np.asarray(x, dtype=np.float32).reshape(-1)]
+    order = sorted(range(len(flat)), key=lambda i: -abs(flat[i]))
+    tau = abs(flat[order[kk - 1]])
+    return np.array([v if abs(v) >= tau else 0.0 for v in flat], dtype=np.float32).reshape(np.shape(x))
+
+
+@pytest.mark.parametrize("shape,frac", [((7, 9), 0.1), ((1, 50), 0.5), ((33, 4), 0.02), ((5, 5), 1.0),
+                                        ((64, 3), 0.005), ((12, 12), 0.25)])
+def test_topk_matches_brute_force_selection(shape, frac):
+    rng = np.random.default_rng(700 + shape[0])
+    x = rng.standard_normal(shape).astype(np.float32)
+    n = x.size
+    kk = min(n, max(1, int(math.floor(float(np.float32(frac)) * n))))
+    assert O.topk_count(n, frac) == kk
+    got = O.topk_sparsify(x, frac)
+    assert np.array_equal(got, _topk_brute(x, kk))
+    kept = got != 0
+    assert kept.sum() == kk                                   # no ties in continuous data
+    assert np.array_equal(got[kept], x[kept])                 # kept entries unchanged, sign included
+    if kk < n:
+        assert np.abs(x[kept]).min() > np.abs(x[~kept]).max() # every kept entry beats every dropped one
+    if frac == 1.0:
+        assert np.array_equal(got, x)
+
+
+def test_topk_is_the_best_k_term_approximation():
+    """Among all arrays with at most kk non-zeros, keeping the kk largest magnitudes is the
+    closest to x in the Frobenius norm: checked by enumerating every support for small n."""
+    import itertools
+    rng = np.random.default_rng(701)
+    for n, frac in [(6, 0.5), (8, 0.25), (7, 0.3), (5, 0.2)]:
+        x = rng.standard_normal(n).astype(np.float32)
+        kk = O.topk_count(n, frac)
+        best = min(float(np.sum(np.delete(x.astype(np.float64), list(sup)) ** 2))
+                   for sup in itertools.combinations(range(n), kk))
+        got = O.topk_sparsify(x.reshape(1, n), frac).reshape(-1)
+        assert np.count_nonzero(got) == kk
+        assert abs(float(np.sum((x.astype(np.float64) - got) ** 2)) - best) < 1e-12
+
+
+def test_topk_ties_counts_and_degenerate_inputs():
+    # ties with the kk-th magnitude are all kept, whatever their sign or position
+    x = np.array([[3.0, -1.0, 1.0, 0.5, -3.0, 1.0, 0.25, -1.0]], dtype=np.float32)
+    assert np.array_equal(O.topk_sparsify(x, 3 / 8), np.array([[3, -1, 1, 0, -3, 1, 0, -1]], dtype=np.float32))
+    assert np.array_equal(O.topk_sparsify(x, 2 / 8), np.array([[3, 0, 0, 0, -3, 0, 0, 0]], dtype=np.float32))
+    # a fraction that selects less than one entry still keeps one; the selection is over the whole tensor,
+    # not per row
+    y = np.array([[1.0, 2.0], [9.0, 3.0], [4.0, 8.0]], dtype=np.float32)
+    assert np.array_equal(O.topk_sparsify(y, 0.01), np.array([[0, 0], [9, 0], [0, 0]], dtype=np.float32))
+    assert np.array_equal(O.topk_sparsify(y, 0.5), np.array([[0, 0], [9, 0], [4, 8]], dtype=np.float32))
+    assert O.topk_count(1000, 0.0005) == 1 and O.topk_count(1000, 0.0025) == 2 and O.topk_count(8, 1.0) == 8
+    # all-zero input stays zero; an empty tensor stays empty
+    assert not O.topk_sparsify(np.zeros((3, 4), np.float32), 0.1).any()
+    assert O.topk_sparsify(np.zeros((0, 4), np.float32), 0.1).shape == (0, 4)
+
+
+def test_sparsified_pseudogradient_definitions_and_error_feedback():
+    rng = np.random.default_rng(702)
+    tg = rng.standard_normal((9, 14)).astype(np.float32)
+    K, frac = 3, 0.2
+    thetas = [(tg - 0.1 * rng.standard_normal(tg.shape)).astype(np.float32) for _ in range(K)]
+    # one worker: Psi is the sparsified delta itself; fraction 1: the plain float32 pseudogradient
+    assert np.array_equal(O.sparsified_pseudogradient(tg, thetas[:1], frac), O.topk_sparsify(tg - thetas[0], frac))
+    assert np.array_equal(O.sparsified_pseudogradient(tg, thetas, 1.0), O.pseudogradient_f32(tg, thetas))
+    # K workers: the mean of the individually sparsified deltas (float64 reference of the same sum)
+    want = sum(O.topk_sparsify(tg - th, frac).astype(np.float64) for th in thetas) / K
+    got = O.sparsified_pseudogradient(tg, thetas, frac)
+    assert np.abs(got - want).max() < 1e-6
+    # error feedback with beta = 1: what was not sent stays in E, entry by entry and exactly
+    # (a kept entry leaves 0 behind, a dropped entry is carried whole)
+    ef = [np.zeros_like(tg) for _ in range(K)]
+    sent_total = [np.zeros(tg.shape, np.float64) for _ in range(K)]
+    delta_total = [np.zeros(tg.shape, np.float64) for _ in range(K)]
+    for rnd in range(4):
+        thetas = [(tg - 0.1 * rng.standard_normal(tg.shape)).astype(np.float32) for _ in range(K)]
+        before = [e.copy() for e in ef]
+        O.sparsified_pseudogradient(tg, thetas, frac, ef, 1.0)
+        for k in range(K):
+            e_in = (before[k] + (tg - thetas[k])).astype(np.float32)
+            sent = O.topk_sparsify(e_in, frac)
+            assert np.array_equal(ef[k], np.where(sent != 0, 0, e_in).astype(np.float32))
+            assert np.count_nonzero(ef[k]) == tg.size - O.topk_count(tg.size, frac)
+            sent_total[k] += sent
+            delta_total[k] += (tg - thetas[k]).astype(np.float32)
+    for k in range(K):
+        assert np.abs(ef[k] + sent_total[k] - delta_total[k]).max() < 1e-5
+    # beta = 0: the accumulator is overwritten, so the sent part equals that of the run without it
+    ef0 = [rng.standard_normal(tg.shape).astype(np.float32) for _ in range(K)]
+    assert np.array_equal(O.sparsified_pseudogradient(tg, thetas, frac, ef0, 0.0),
+                          O.sparsified_pseudogradient(tg, thetas, frac))
+
+
+def test_oracle_sync_with_topk_runs_algorithm_2():
+    rng = np.random.default_rng(703)
+    specs = [O.TensorSpec("a", 6, 10), O.TensorSpec("b", 1, 17, kind="adamw")]
+    init = [rng.standard_normal((s.rows, s.cols)).astype(np.float32) for s in specs]
+    cfg = O.OracleConfig(K=2, H=1, outer_lr=0.5, outer_momentum=0.0, topk_fraction=0.25, error_feedback=True)
+    orc = O.MuLoCoOracle(cfg, specs, init)
+    for k in range(2):
+        for i in range(2):
+            orc.theta_k[k][i] += rng.standard_normal(init[i].shape).astype(np.float32)
+    tg0 = [w.copy() for w in orc.theta_g]
+    d = [[(tg0[i] - orc.theta_k[k][i]).astype(np.float32) for i in range(2)] for k in range(2)]
+    orc.outer_sync()
+    for i in range(2):
+        psi = (O.topk_sparsify(d[0][i], 0.25).astype(np.float64) + O.topk_sparsify(d[1][i], 0.25)) / 2
+        assert np.abs(orc.theta_g[i] - (tg0[i] - 0.5 * psi)).max() < 1e-6     # mu = 0: plain SGD outer step
+        assert np.array_equal(orc.theta_k[0][i], orc.theta_g[i])
+        assert np.count_nonzero(orc.ef[0][i]) == init[i].size - O.topk_count(init[i].size, 0.25)
+    with pytest.raises(ValueError):
+        O.MuLoCoOracle(O.OracleConfig(K=2, H=1, topk_fraction=0.1, quant_bits=8), specs, init)
