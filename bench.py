@@ -237,7 +237,9 @@ def main():
     ap.add_argument("--quant-stages", type=int, default=1, help="with --sync-only: 2 = per-worker quantisation + "
                     "second quantisation of the mean (Algorithm 2)")
     ap.add_argument("--quant-block", type=int, default=128, help="with --sync-only: 32/64/128, or 0 = row-wise")
-    ap.add_argument("--ef", action="store_true", help="with --sync-only --quant-stages 2: error feedback")
+    ap.add_argument("--ef", action="store_true", help="with --sync-only --quant-stages 2 or --topk: error feedback")
+    ap.add_argument("--topk", type=float, default=0.0, help="with --sync-only (QUANT 0): top-k sparsification of "
+                    "every worker's delta, the fraction kept")
     ap.add_argument("--adamw-only", type=int, nargs=2, metavar=("K", "MPARAMS"), default=None,
                     help="kernel study: time the AdamW part of muloco_inner_step on MPARAMS million parameters")
     ap.add_argument("--muon-only", type=int, nargs=4, metavar=("K", "LAYERS", "D", "F"), default=None,
@@ -490,7 +492,7 @@ def run_elementwise_only(args):
     w = configs.Workload("elementwise-only", K=K, H=1, J=1, tensors=ts, muon_lr=0.02, muon_beta=0.9, muon_wd=0.01,
                          outer_lr=0.7, outer_momentum=0.9, quant_bits=quant,
                          quant_stages=args.quant_stages if sync else 1, error_feedback=bool(args.ef and sync),
-                         quant_block=args.quant_block)
+                         quant_block=args.quant_block, topk_fraction=args.topk if sync else 0.0)
     opt = binding.MuLoCo(w, "cuda:0", init_seed=1, alloc_grads=not sync)
     gen = torch.Generator(device="cuda"); gen.manual_seed(0)
     if sync:
@@ -515,11 +517,14 @@ def run_elementwise_only(args):
     if sync:
         ms = ph["sync"] / args.steps
         nbytes = n * ((16.0 if args.ef else 8.0) * K + 16.0)      # error feedback: K more reads and writes
+        if args.topk > 0:                                         # three histogram passes read theta and every delta
+            nbytes += n * 3 * ((8.0 if args.ef else 4.0) * K + 4.0)
     else:
         ms = ph["adamw"] / args.steps
         nbytes = n * K * 28.0
     gbs = nbytes / (ms * 1e-3) / 1e9
-    print(json.dumps({"sync_only" if sync else "adamw_only": [K, mparams, quant], "params": n, "ms_per_call": ms,
+    print(json.dumps({"sync_only" if sync else "adamw_only": [K, mparams, quant], "topk": args.topk, "params": n,
+                      "ms_per_call": ms,
                       "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "launches": int(launches)}))
     opt.close()
 

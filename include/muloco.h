@@ -97,9 +97,18 @@ typedef struct {
                            again                                                            */
   uint64_t workspace_bytes; /* Newton-Schulz workspace budget; 0 lets the library pick  */
   int32_t error_feedback; /* 1: Algorithm 2's error feedback, E_i <- beta E_i + Delta_i,
-                             send C(E_i), E_i <- E_i - C(E_i); needs quant_stages == 2 and
-                             the ef_k buffers                                              */
+                             send C(E_i), E_i <- E_i - C(E_i); needs the ef_k buffers and a
+                             per-worker compressor: quant_stages == 2 with a quantiser, or
+                             topk_fraction > 0                                              */
   float ef_beta;       /* beta of the error-feedback accumulator                          */
+  float topk_fraction; /* 0: off.  In (0, 1]: top-k sparsification (Section 2, "Compressed
+                          Communication") of every worker's delta, per tensor: with n elements,
+                          kk = max(1, floor(topk_fraction * n)) (in double), the entries whose
+                          magnitude is at least the kk-th largest are kept (ties all kept), the
+                          rest become 0; the mean of the sparsified deltas is the
+                          pseudogradient, nothing is compressed after the mean.  Needs
+                          quant == MULOCO_Q_NONE; error_feedback may be set with it.  Tensors
+                          of 2^31 elements or more make muloco_create return MULOCO_ESHAPE.    */
 } muloco_config;
 
 /* State buffers.  Every field is a HOST array of DEVICE pointers.
@@ -230,6 +239,13 @@ MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, float* O, i
  * bits is 8, 4 or 2. */
 MULOCO_API muloco_status muloco_quantize(muloco_ctx* ctx, const float* psi, int64_t rows, int64_t cols,
                               int32_t bits, int8_t* codes, float* scales, float* dequant);
+
+/* The top-k sparsifier on its own (Section 2, "Compressed Communication"): x and out are
+ * DEVICE arrays of n float32 (they may be the same array); out = x where |x| is at least the
+ * kk-th largest magnitude, kk = max(1, floor(fraction * n)), else 0.  fraction in (0, 1].
+ * Allocates and frees a few KB of device scratch; waits for the stream before returning. */
+MULOCO_API muloco_status muloco_topk_sparsify(muloco_ctx* ctx, const float* x, int64_t n, float fraction,
+                                   float* out);
 
 /* Test hook: the pseudogradient of tensor `tensor` (Eq. 2), exactly as
  * muloco_outer_sync forms it, written to psi_out (float32, tensor's shape),

@@ -30,7 +30,7 @@ PHASES = ["prologue", "ns", "adamw", "sync", "copy"]
 EXPORTS = [
     "muloco_create", "muloco_destroy", "muloco_inner_step", "muloco_inner_step_host",
     "muloco_outer_sync", "muloco_outer_sync_host", "muloco_fragments_due", "muloco_newton_schulz",
-    "muloco_quantize", "muloco_pseudogradient", "muloco_get_state", "muloco_set_state",
+    "muloco_quantize", "muloco_topk_sparsify", "muloco_pseudogradient", "muloco_get_state", "muloco_set_state",
     "muloco_set_timing", "muloco_get_timings", "muloco_sync_status", "muloco_last_error",
     "muloco_newton_schulz_static",
 ]
@@ -52,7 +52,8 @@ class Config(C.Structure):
                 ("outer_lr", C.c_float), ("outer_momentum", C.c_float),
                 ("quant", C.c_int32), ("quant_block", C.c_int32), ("grad_dtype", C.c_int32),
                 ("quant_stages", C.c_int32), ("workspace_bytes", C.c_uint64),
-                ("error_feedback", C.c_int32), ("ef_beta", C.c_float)]
+                ("error_feedback", C.c_int32), ("ef_beta", C.c_float),
+                ("topk_fraction", C.c_float)]
 
 
 class Buffers(C.Structure):
@@ -92,6 +93,7 @@ def load_library():
     lib.muloco_newton_schulz.argtypes = [vp, vp, i32, vp, i32, i32, i64, i64, i32]
     lib.muloco_quantize.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
     lib.muloco_pseudogradient.argtypes = [vp, i32, vp]
+    lib.muloco_topk_sparsify.argtypes = [vp, vp, i64, C.c_float, vp]
     lib.muloco_get_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
     lib.muloco_set_state.argtypes = [vp, vp, C.c_size_t]
     lib.muloco_set_timing.argtypes = [vp, i32]
@@ -150,6 +152,7 @@ def make_config(w: _cfg.Workload, workspace_bytes: int = 0, ns_mode: Optional[st
     c.quant_stages = w.quant_stages
     c.error_feedback = int(w.error_feedback)
     c.ef_beta = w.ef_beta
+    c.topk_fraction = w.topk_fraction
     c.grad_dtype = BF16 if w.grad_dtype == "bf16" else F32
     c.workspace_bytes = workspace_bytes
     for k, v in over.items():
@@ -353,6 +356,13 @@ class MuLoCo:
         self._check(self.lib.muloco_quantize(self.ctx, p.data_ptr(), rows, cols, bits, codes.data_ptr(),
                                              scales.data_ptr(), deq.data_ptr()))
         return codes, scales, deq
+
+    def topk_sparsify(self, x, fraction: float):
+        torch = self.torch
+        xc = x.contiguous()
+        out = torch.empty_like(xc)
+        self._check(self.lib.muloco_topk_sparsify(self.ctx, xc.data_ptr(), xc.numel(), fraction, out.data_ptr()))
+        return out
 
     def pseudogradient(self, tensor: int):
         torch = self.torch

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmuloco.so")
-SOURCES = ["capi.cu", "elementwise.cu", "outer_sync.cu", "ns_fp32.cu", "ns_tc.cu", "ns_static.cu"]
+SOURCES = ["capi.cu", "elementwise.cu", "outer_sync.cu", "topk.cu", "ns_fp32.cu", "ns_tc.cu", "ns_static.cu"]
 
 
 def _nvcc() -> str:

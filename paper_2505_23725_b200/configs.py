@@ -45,8 +45,9 @@ class Workload:
     quant_bits: int = 0                 # 0 (none), 8, 4 or 2
     quant_block: int = 128
     quant_stages: int = 1               # 2: per-worker quantisation, fp32 mean, second quantisation
-    error_feedback: bool = False        # Algorithm 2's accumulators (needs quant_stages = 2)
+    error_feedback: bool = False        # Algorithm 2's accumulators (needs quant_stages = 2 or top-k)
     ef_beta: float = 1.0
+    topk_fraction: float = 0.0          # > 0: top-k sparsification of every worker's delta
     adam_lr: Optional[float] = None     # None: same as muon_lr
     adam_wd: Optional[float] = None     # None: same as muon_wd
     adam_beta1: float = 0.9

@@ -44,7 +44,15 @@ struct Group {
   TcGroupPlan* plan = nullptr;
 };
 
+// How many entries top-k keeps of n: floor(fraction * n) in double, at least 1, at most n.
+uint32_t topk_keep(int64_t n, float fraction) {
+  int64_t kk = (int64_t)floor((double)fraction * (double)n);
+  kk = std::max<int64_t>(1, std::min<int64_t>(kk, n));
+  return (uint32_t)kk;
+}
+
 struct FragTable {
+  uint32_t* d_kk = nullptr;     // top-k: entries kept per segment
   SyncSeg* d_segs = nullptr;
   int n_segs = 0;
   int64_t n_units = 0;
@@ -101,6 +109,7 @@ struct muloco_ctx {
   std::vector<FragTable> frags;   // J entries + one for "all"
   float** d_replicas = nullptr;   // [n][K]
   float** d_ef = nullptr;         // [n][K] error-feedback accumulators (Algorithm 2), or NULL
+  TopkScratch topk;               // radix-select scratch, [n][K] problems (top-k only)
 
   // per-call tables
   MatDesc* d_mats = nullptr;
@@ -201,8 +210,13 @@ muloco_status validate_config(const muloco_config* cfg) {
     return fail(c, MULOCO_EINVAL, "quant must be 0, 2, 4 or 8");
   if (cfg->quant_stages < 0 || cfg->quant_stages > 2)
     return fail(c, MULOCO_EINVAL, "quant_stages must be 0, 1 or 2");
-  if (cfg->error_feedback != 0 && (cfg->quant_stages != 2 || cfg->quant == MULOCO_Q_NONE))
-    return fail(c, MULOCO_EINVAL, "error_feedback needs quant_stages == 2 and a quantiser");
+  if (!(cfg->topk_fraction >= 0.f && cfg->topk_fraction <= 1.f))
+    return fail(c, MULOCO_EINVAL, "topk_fraction must be in [0, 1]");
+  if (cfg->topk_fraction > 0.f && cfg->quant != MULOCO_Q_NONE)
+    return fail(c, MULOCO_EINVAL, "top-k sparsification and quantisation are not combined");
+  if (cfg->error_feedback != 0 && !(cfg->topk_fraction > 0.f) &&
+      (cfg->quant_stages != 2 || cfg->quant == MULOCO_Q_NONE))
+    return fail(c, MULOCO_EINVAL, "error_feedback needs quant_stages == 2 and a quantiser, or topk_fraction > 0");
   if (cfg->error_feedback != 0 && !(cfg->ef_beta >= 0.f && cfg->ef_beta <= 1.f))
     return fail(c, MULOCO_EINVAL, "ef_beta must be in [0, 1]");
   if (!valid_block(cfg->quant_block)) return fail(c, MULOCO_EINVAL, "quant_block must be 0 (row-wise), 32, 64 or 128");
@@ -302,10 +316,25 @@ muloco_status build_sync_tables(muloco_ctx* c) {
       CK(cudaMemcpy(c->d_ef, reps.data(), reps.size() * sizeof(float*), cudaMemcpyHostToDevice));
     }
   }
+  const bool topk = c->cfg.topk_fraction > 0.f;
+  if (topk && n > 0) {
+    for (int i = 0; i < n; ++i)
+      if (c->T[i].numel() >= ((int64_t)1 << 31))
+        return fail(c, MULOCO_ESHAPE, "top-k: tensor %d has 2^31 elements or more", i);
+    const size_t problems = (size_t)n * K;
+    const size_t hist_bytes = problems * topk_hist_words_per_problem() * sizeof(uint32_t);
+    CK(cudaMalloc(&c->topk.hist, hist_bytes));
+    CK(cudaMalloc(&c->topk.prefix, problems * sizeof(uint32_t)));
+    CK(cudaMalloc(&c->topk.remaining, problems * sizeof(uint32_t)));
+    CK(cudaMemsetAsync(c->topk.hist, 0, hist_bytes, c->st));
+    CK(cudaMemsetAsync(c->topk.prefix, 0, problems * sizeof(uint32_t), c->st));
+    CK(cudaMemsetAsync(c->topk.remaining, 0, problems * sizeof(uint32_t), c->st));
+  }
   c->frags.resize(c->cfg.J + 1);
   for (int f = 0; f <= c->cfg.J; ++f) {
     FragTable& ft = c->frags[f];
     std::vector<SyncSeg> segs;
+    std::vector<uint32_t> kks;
     int64_t units = 0;
     for (int i = 0; i < n; ++i) {
       const TensorInfo& t = c->T[i];
@@ -323,12 +352,17 @@ muloco_status build_sync_tables(muloco_ctx* c) {
       s.rep_index = (int64_t)i * K;
       units += s.rows * s.nblk;
       segs.push_back(s);
+      if (topk) kks.push_back(topk_keep(t.numel(), c->cfg.topk_fraction));
     }
     ft.n_segs = (int)segs.size();
     ft.n_units = units;
     if (!segs.empty()) {
       CK(cudaMalloc(&ft.d_segs, segs.size() * sizeof(SyncSeg)));
       CK(cudaMemcpy(ft.d_segs, segs.data(), segs.size() * sizeof(SyncSeg), cudaMemcpyHostToDevice));
+      if (topk) {
+        CK(cudaMalloc(&ft.d_kk, kks.size() * sizeof(uint32_t)));
+        CK(cudaMemcpy(ft.d_kk, kks.data(), kks.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
+      }
     }
   }
   return MULOCO_OK;
@@ -508,7 +542,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
     CKC(cudaMemcpy(c->d_wmaps, hmaps.data(), hmaps.size(), cudaMemcpyHostToDevice));
   }
 
-  if (build_sync_tables(c) != MULOCO_OK) return bail(MULOCO_ECUDA);
+  { const muloco_status bs = build_sync_tables(c); if (bs != MULOCO_OK) return bail(bs); }
 
   // Algorithm 1, initialisation: u <- 0, inner state <- 0, theta_k <- theta_g
   for (int i = 0; i < n_tensors; ++i) {
@@ -538,6 +572,9 @@ MULOCO_API void muloco_destroy(muloco_ctx* c) {
   if (c->d_status) cudaFree(c->d_status);
   if (c->d_replicas) cudaFree(c->d_replicas);
   if (c->d_ef) cudaFree(c->d_ef);
+  if (c->topk.hist) cudaFree(c->topk.hist);
+  if (c->topk.prefix) cudaFree(c->topk.prefix);
+  if (c->topk.remaining) cudaFree(c->topk.remaining);
   if (c->d_mats) cudaFree(c->d_mats);
   if (c->d_adam) cudaFree(c->d_adam);
   if (c->d_wmaps) cudaFree(c->d_wmaps);
@@ -549,8 +586,10 @@ MULOCO_API void muloco_destroy(muloco_ctx* c) {
   if (c->copy_st) cudaStreamDestroy(c->copy_st);
   if (c->copy_st2) cudaStreamDestroy(c->copy_st2);
   if (c->stage) cudaFree(c->stage);
-  for (FragTable& f : c->frags)
+  for (FragTable& f : c->frags) {
     if (f.d_segs) cudaFree(f.d_segs);
+    if (f.d_kk) cudaFree(f.d_kk);
+  }
   for (int r = 0; r < RING; ++r) {
     if (c->h_ring[r]) cudaFreeHost(c->h_ring[r]);
     if (c->ring_ev[r]) cudaEventDestroy(c->ring_ev[r]);
@@ -746,6 +785,12 @@ MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* c, int32_t fragment) {
   if (fragment < 0) for (auto& s : c->frag_syncs) s += 1; else c->frag_syncs[fragment] += 1;
   if (ft.n_segs == 0) return MULOCO_OK;
   PhaseTimer t(c, MULOCO_PH_SYNC);
+  if (f.topk_fraction > 0.f) {
+    c->launches += launch_outer_sync_topk(c->st, ft.d_segs, ft.n_segs, c->d_replicas, f.K, ft.n_units, f.outer_lr,
+                                          f.outer_momentum, c->d_status, c->d_ef, f.ef_beta, ft.d_kk, c->topk);
+    CK(cudaGetLastError());
+    return MULOCO_OK;
+  }
   const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
   if (f.quant != MULOCO_Q_NONE && blk == 0) {
     cudaError_t e = launch_outer_sync_rows(c->st, ft.d_segs, ft.n_segs, c->d_replicas, f.K, ft.n_units, ft.max_cols,
@@ -871,6 +916,40 @@ MULOCO_API muloco_status muloco_quantize(muloco_ctx* c, const float* psi, int64_
   launch_quantize(c->st, psi, rows, cols, c->cfg.quant_block, bits, codes, scales, dequant, c->d_status);
   c->launches += 1;
   CK(cudaGetLastError());
+  return MULOCO_OK;
+}
+
+MULOCO_API muloco_status muloco_topk_sparsify(muloco_ctx* c, const float* x, int64_t n, float fraction, float* out) {
+  if (!c) return MULOCO_EINVAL;
+  if (!(fraction > 0.f && fraction <= 1.f)) return fail(c, MULOCO_EINVAL, "fraction must be in (0, 1]");
+  if (n < 0 || n >= ((int64_t)1 << 31)) return fail(c, MULOCO_ESHAPE, "n must be in 0..2^31-1");
+  if (n == 0) return MULOCO_OK;                      // empty input: nothing to read or write
+  if (!x || !out) return fail(c, MULOCO_EINVAL, "x or out is NULL");
+  const size_t words = topk_hist_words_per_problem() + 4;
+  char* scratch = nullptr;
+  CK(cudaMalloc(&scratch, words * sizeof(uint32_t) + sizeof(SyncSeg)));
+  uint32_t* w = reinterpret_cast<uint32_t*>(scratch);
+  TopkScratch sc;
+  sc.hist = w;
+  sc.prefix = w + topk_hist_words_per_problem();
+  sc.remaining = sc.prefix + 1;
+  uint32_t* d_kk = sc.prefix + 2;
+  SyncSeg* d_seg = reinterpret_cast<SyncSeg*>(scratch + words * sizeof(uint32_t));
+  SyncSeg seg;
+  seg.theta_g = const_cast<float*>(x); seg.u = nullptr;
+  seg.rows = 1; seg.cols = n; seg.nblk = (n + 127) / 128; seg.unit_begin = 0; seg.rep_index = 0;
+  const uint32_t kk = topk_keep(n, fraction);
+  cudaError_t e = cudaMemsetAsync(scratch, 0, words * sizeof(uint32_t), c->st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_kk, &kk, sizeof kk, cudaMemcpyHostToDevice, c->st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_seg, &seg, sizeof seg, cudaMemcpyHostToDevice, c->st);
+  if (e == cudaSuccess) {
+    c->launches += launch_topk_raw(c->st, d_seg, n, x, out, d_kk, sc, c->d_status);
+    e = cudaGetLastError();
+  }
+  const cudaError_t e2 = cudaStreamSynchronize(c->st);   // kk and seg are stack variables; scratch is freed below
+  cudaFree(scratch);
+  CK(e);
+  CK(e2);
   return MULOCO_OK;
 }
 

@@ -107,6 +107,24 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
 cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
                                    int K, int64_t n_rows, int64_t max_cols, int quant_bits, float outer_lr,
                                    float mu, int* status, int stages, float* const* ef, float ef_beta);
+// Top-k sparsification of the workers' deltas (topk.cu).  Scratch: one histogram of
+// topk_hist_words_per_problem() words (zero between calls), one prefix word (the threshold key
+// after a call) and one counter per (tensor, worker), indexed like the replica table.
+// kk_seg[i] = how many entries segment i keeps.  Segments are flat (rows == 1, 128-element units).
+// Returns the number of kernels launched.
+struct TopkScratch {
+  uint32_t* hist = nullptr;
+  uint32_t* prefix = nullptr;
+  uint32_t* remaining = nullptr;
+};
+size_t topk_hist_words_per_problem();
+int launch_outer_sync_topk(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,
+                           int64_t n_units, float outer_lr, float mu, int* status, float* const* ef,
+                           float ef_beta, const uint32_t* kk_seg, TopkScratch sc);
+// Standalone: out = top-k(x) for one device array of n elements; seg_dev describes x as one flat
+// segment (theta_g = x, rep_index = 0), kk_dev holds the count to keep.
+int launch_topk_raw(cudaStream_t st, const SyncSeg* seg_dev, int64_t n, const float* x, float* out,
+                    const uint32_t* kk_dev, TopkScratch sc, int* status);
 void launch_pseudogradient(cudaStream_t st, const float* theta_g, float* const* replicas, int K,
                            int64_t n, float* psi_out);
 void launch_quantize(cudaStream_t st, const float* psi, int64_t rows, int64_t cols, int block,
