@@ -23,7 +23,8 @@ namespace {
 constexpr int TK_THREADS = 256;
 constexpr int TK_WARPS = TK_THREADS / 32;
 constexpr int TK_UNIT = 128;                // elements per warp step (4 per lane)
-constexpr int TK_UNITS_PER_CTA = 64;        // histogram passes: 8192 elements per CTA and worker
+constexpr int TK_UNITS_PER_CTA = 256;       // histogram passes: 32768 elements per CTA and worker (measured: 26.4 ms
+                                            // per sync of 400M parameters x 16 workers, against 28.8 with 64 and 32.2 with 32)
 constexpr int TK_APPLY_UNITS_PER_CTA = 32;  // fused pass: small CTAs in address order
 constexpr int TK_BINS = 2048;               // widest digit (11 bits)
 

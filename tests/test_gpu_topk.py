@@ -173,3 +173,38 @@ def test_topk_configuration_errors_and_nonfinite_delta():
         gpu.sync_status()
     assert e.value.status == binding.ENONFINITE
     gpu.close()
+
+
+def test_topk_sync_at_benchmark_shapes():
+    """The 416M-shaped model's tensor shapes (embedding and head of 32000 x 1024, hidden matrices of
+    1024 x 1024, 1024 x 2816 and 2816 x 1024, gain vectors) with two layers and K = 4: one sync with
+    top-k and error feedback; the oracle recomputes one tensor of every distinct shape in full."""
+    import torch
+    from paper_2505_23725_b200 import binding
+    K, frac = 4, 0.01
+    ts = configs.llama_tensors(2, 1024, 2816, vocab=32000, norms=True)
+    w = configs.Workload("topk-416M-shapes", K=K, H=1, J=1, tensors=ts, muon_lr=0.02, muon_beta=0.9, muon_wd=0.0,
+                         outer_lr=0.7, outer_momentum=0.9, topk_fraction=frac, error_feedback=True, ef_beta=0.9)
+    opt = binding.MuLoCo(w, "cuda:0", init_seed=11, alloc_grads=False)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(3)
+    for k in range(K):
+        opt.flat_theta_k[k].add_(torch.empty_like(opt.flat_theta_k[k]).normal_(0.0, 1e-3, generator=gen))
+        opt.flat_ef[k].normal_(0.0, 1e-4, generator=gen)
+    opt.flat_u.normal_(0.0, 1e-3, generator=gen)
+    first = {}
+    for i, t in enumerate(ts):
+        first.setdefault((t.rows, t.cols), i)
+    sample = sorted(first.values())
+    snap = {i: (_np(opt.theta_g[i]).copy(), _np(opt.outer_u[i]).copy(), [_np(opt.theta_k[k][i]).copy() for k in range(K)],
+                [_np(opt.ef[k][i]).copy() for k in range(K)]) for i in sample}
+    opt.outer_sync(-1)
+    opt.sync_status()
+    for i, (tg, u, reps, efs) in snap.items():
+        psi = O.sparsified_pseudogradient(tg, reps, frac, efs, 0.9)
+        O.outer_nesterov(tg, u, psi, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum)
+        for k in range(K):
+            assert np.array_equal(_np(opt.ef[k][i]), efs[k]), f"E k={k} {ts[i].name}"
+        assert_close_1e6(_np(opt.theta_g[i]), tg, f"theta_g {ts[i].name}")
+        assert_close_1e6(_np(opt.outer_u[i]), u, f"u {ts[i].name}")
+        assert np.array_equal(_np(opt.theta_k[K - 1][i]), _np(opt.theta_g[i]))
+    opt.close()
