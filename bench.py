@@ -501,7 +501,16 @@ def run_elementwise_only(args):
     else:
         for k in range(K):
             opt.flat_grads[k].normal_(0.0, 0.01, generator=gen)
-    call = (lambda: opt.outer_sync(-1)) if sync else (lambda: opt.inner_step(-1, None, 1.0))
+    def sync_call():
+        # a sync leaves theta_k = theta, so without new drift every later delta would be zero; the
+        # radix select of top-k depends on the data, so the replicas drift again before every call
+        # (outside the timed span: the phase timer brackets the library's own launches only)
+        if args.topk > 0:
+            for k in range(K):
+                opt.flat_theta_k[k].add_(noise.normal_(0.0, 1e-3, generator=gen))
+        opt.outer_sync(-1)
+    noise = torch.empty_like(opt.flat_theta_g) if sync and args.topk > 0 else None
+    call = sync_call if sync else (lambda: opt.inner_step(-1, None, 1.0))
     for _ in range(args.warmup):
         call()
     opt.set_timing(True); opt.get_timings()

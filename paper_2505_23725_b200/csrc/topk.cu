@@ -123,23 +123,28 @@ topk_hist_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __r
         if (MODE == 1) tk_load4(ep + off, vec, nvalid, e);
       }
       form_x<MODE>(tg, r, e, ef_beta, x);
+      uint32_t dg[4];
+      bool in[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const uint32_t key = mag_key(x[q]);
-        const bool in = (q < nvalid) && (PASS == 0 || (key >> (SH + digit_bits(PASS))) == pre);
-        const uint32_t dg = (key >> SH) & (uint32_t)(NB - 1);
-        if (PASS == 0) {
-          // the leading digit is the exponent: most lanes hit a handful of bins, so count equal
-          // digits within the warp first
-          const unsigned act = __ballot_sync(0xffffffffu, in);
-          if (in) {
-            const unsigned same = __match_any_sync(act, dg);
-            if ((__ffs(same) - 1) == lane) atomicAdd(&hist[dg], (uint32_t)__popc(same));
-          }
-        } else if (in) {
-          atomicAdd(&hist[dg], 1u);
+        in[q] = (q < nvalid) && (PASS == 0 || (key >> (SH + digit_bits(PASS))) == pre);
+        dg[q] = (key >> SH) & (uint32_t)(NB - 1);
+      }
+      if (PASS == 0) {
+        // The leading digit is the exponent.  A full unit whose 128 keys share it (zero deltas, a
+        // constant tensor) adds once; otherwise plain shared-memory atomics: a warp's keys fall
+        // into a few dozen bins, a few lanes per bin.
+        const uint32_t d0 = __shfl_sync(0xffffffffu, dg[0], 0);
+        const bool same = nvalid == 4 && dg[0] == d0 && dg[1] == d0 && dg[2] == d0 && dg[3] == d0;
+        if (__all_sync(0xffffffffu, same)) {
+          if (lane == 0) atomicAdd(&hist[d0], (uint32_t)TK_UNIT);
+          continue;
         }
       }
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (in[q]) atomicAdd(&hist[dg[q]], 1u);
     }
     __syncthreads();
     uint32_t* gh = ghist + problem * TK_BINS;
