@@ -74,6 +74,19 @@ class Workload:
                 f += 5.0 * (4.0 * s * s * l + 2.0 * s ** 3)
         return f * self.K
 
+    def ns_flops_executed(self) -> float:
+        """What the tensor-core engine multiplies: the two symmetric products of an iteration (Gram,
+        polynomial) run only the tiles on and above the diagonal -- T(T+1)/2 of T^2 tiles of 256 rows
+        (one tile for matrices of up to 128 rows) -- the third product runs in full."""
+        f = 0.0
+        for t in self.tensors:
+            if t.kind == MUON:
+                s, l = min(t.rows, t.cols), max(t.rows, t.cols)
+                T = 1 if s <= 128 else -(-s // 256)
+                tri = (T + 1) / (2.0 * T)
+                f += 5.0 * (tri * 2.0 * s * s * l + tri * 2.0 * s ** 3 + 2.0 * s * s * l)
+        return f * self.K
+
     def sync_bytes(self, fragment: int = -1) -> float:
         """(8K + 16) bytes per parameter of the fragment: K+2 fp32 reads and K+2 fp32 writes."""
         n = sum(t.numel for t in self.tensors if fragment < 0 or t.fragment == fragment)
