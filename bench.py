@@ -243,6 +243,7 @@ def main():
                     "every worker's delta, the fraction kept")
     ap.add_argument("--adamw-only", type=int, nargs=2, metavar=("K", "MPARAMS"), default=None,
                     help="kernel study: time the AdamW part of muloco_inner_step on MPARAMS million parameters")
+    ap.add_argument("--grad-dtype", choices=["f32", "bf16"], default="f32", help="with --muon-only: gradient type")
     ap.add_argument("--muon-only", type=int, nargs=4, metavar=("K", "LAYERS", "D", "F"), default=None,
                     help="kernel study: muloco_inner_step on LAYERS layers of hidden matrices only "
                          "(prologue + Newton-Schulz with the fused parameter update), K workers")
@@ -458,7 +459,7 @@ def run_muon_only(args):
     entry.build()
     K, L, d, F = args.muon_only
     w = configs.mini_workload(K=K, H=1, J=1, ns_mode="bf16", L=L, d=d, F=F, muon_lr=4.42e-2, muon_beta=0.9,
-                              muon_wd=6.25e-4)
+                              muon_wd=6.25e-4, grad_dtype=args.grad_dtype)
     opt = binding.MuLoCo(w, "cuda:0", init_seed=1, alloc_grads=True,
                          workspace_bytes=int(args.workspace_gb * (1 << 30)))
     synth.torch_fill_gradients(opt.grads, w.tensors, w.K, 3, opt.device)
@@ -475,7 +476,10 @@ def run_muon_only(args):
     peaks = load_peaks()
     tf = w.ns_flops_credited() / (ph["ns"] / args.steps * 1e-3) / 1e12
     print(json.dumps({"muon_only": [K, L, d, F], "params_per_replica": w.n_params, "ns_ms": ph["ns"] / args.steps,
-                      "prologue_ms": ph["prologue"] / args.steps, "ns_tflops_credited": tf,
+                      "prologue_ms": ph["prologue"] / args.steps,
+                      "prologue_gbs": w.n_params * K * (14.0 if args.grad_dtype == "f32" else 12.0)
+                      / (ph["prologue"] / args.steps * 1e-3) / 1e9,
+                      "ns_tflops_credited": tf,
                       "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"], "launches": int(launches)}))
     opt.close()
 
