@@ -6,9 +6,9 @@
 // (Section 2, "Muon": X_j = p(X X^T) X, p(x) = a x + b x^3 + c x^5) for every
 // matrix of a chunk; tiles of all matrices form one linear work list:
 //   GRAM  : A  = r^2 X X^T      symmetric: only the tiles on or above the diagonal are computed
-//   POLY  : B  = b A + c A A    AND stored; a consumer fetches a block below the diagonal as the
-//                               transpose of its mirror image (an MN-major operand)
-//   APPLY : X' = r (a X + B X)
+//   POLY  : B' = a I + b A + c A A   AND stored; a consumer fetches a block below the diagonal as
+//                               the transpose of its mirror image (an MN-major operand)
+//   APPLY : X' = r B' X  (= r (a X + b A X + c A A X); with a on B's diagonal the product needs no addend)
 //   FINAL : as APPLY, result goes to the parameter update / output sink
 // Operand forms: GRAM/POLY multiply a row-major matrix by its own transpose
 // (both operands K-major); APPLY needs X with the contraction index as the slow
@@ -27,7 +27,7 @@
 // (rank 0) issues the MMAs, warps 2-5 run the epilogue (one 32-lane quarter of
 // the accumulator each).  Two accumulators alternate so the epilogue of one
 // tile overlaps the main loop of the next.  The epilogue goes through shared
-// memory: the addend (A for POLY, X for APPLY) arrives by TMA, results leave as
+// memory: the addend (A for POLY) arrives by TMA, results leave as
 // bulk tensor stores of whole 32 x 64 blocks (and, for the symmetric products,
 // of the transposed block), so global memory only sees full lines.
 // Every wait is bounded: when one runs out the kernel raises ST_TIMEOUT, all
@@ -49,14 +49,13 @@ constexpr int BM = 128;          // rows per CTA (one CTA's share of UMMA M)
 constexpr int BK = 64;           // k slab per stage (64 bf16 = one 128-byte swizzle row)
 constexpr int UMMA_K = 16;
 constexpr int TC_THREADS = 192;
-// Pipeline depth is a template parameter: products that need all six staging blocks per epilogue
-// warp (FINAL: addend + parameter ring) run 4 stages, those that need at most four (GRAM: results;
-// POLY, APPLY: addend + results) run 5 in the same shared memory.
+// Pipeline depth is a template parameter; every product runs 5 stages beside four staging blocks
+// per epilogue warp (GRAM, APPLY: results; POLY: addend + results; FINAL: the parameter ring).
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;        // 16 KB: 128 rows x 64 k
 constexpr uint32_t B_STAGE_BYTES = 128 * BK * 2;       // 16 KB: this CTA's 128 columns of the right operand
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr uint32_t EPI_BLOCK_BYTES = 32 * 64 * 2;      // one 32 x 64 bf16 block
-__host__ __device__ constexpr uint32_t epi_warp_bytes(int nstg) { return (nstg == 5 ? 4u : 6u) * EPI_BLOCK_BYTES; }
+__host__ __device__ constexpr uint32_t epi_warp_bytes(int) { return 4u * EPI_BLOCK_BYTES; }
 __host__ __device__ constexpr uint32_t smem_bytes(int nstg) {
   return (uint32_t)nstg * STAGE_BYTES + 4u * epi_warp_bytes(nstg) + 1024u;   // + alignment slack
 }
@@ -272,7 +271,7 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
 // ------------------------------- the kernel --------------------------------
 // tmA/tmB : operand loads (left: K-major 64 x 128 boxes; right: K-major 64 x 128 or, for B_MN,
 //           MN-major 64 x 64 boxes)
-// tmC     : addend loads, 64 x 32 boxes (POLY: A, APPLY/FINAL: X)
+// tmC     : addend loads, 64 x 32 boxes (POLY: A; unused by the other products)
 // tmD     : result stores, 64 x 32 boxes, 128-byte swizzle
 // tmS     : 64 x 64 boxes over the symmetric operand (POLY: A, APPLY/FINAL: B) for the k slabs
 //           whose block lies below the diagonal and is read from its mirror image
@@ -458,11 +457,13 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     auto out_buf = [&](uint32_t b) { return epi + (o_first + b) * EPI_BLOCK_BYTES; };
     const uint32_t cin_bar0 = smem_u32(&bar_cin[ew][0]);
     auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
-    const bool has_cin = (p.kind != GEMM_GRAM);
+    // Only the polynomial has an addend (b A).  Its epilogue also adds a to the diagonal, B' = B + a I,
+    // so that the third product of the iteration, a X + B X = B' X, needs none.
+    const bool has_cin = (p.kind == GEMM_POLY);
     const bool stores = (p.kind != GEMM_FINAL);
-    // parameter update through TMA: a ring of four 32 x 32 fp32 blocks in the staging space that
-    // after the addend blocks (the final product stages no results)
-    auto w_buf = [&](uint32_t b) { return epi + (2u + b) * EPI_BLOCK_BYTES; };
+    // parameter update through TMA: a ring of four 32 x 32 fp32 blocks, the whole staging space of
+    // the warp (the final product has no addend and stages no results)
+    auto w_buf = [&](uint32_t b) { return epi + b * EPI_BLOCK_BYTES; };
     const uint32_t w_bar0 = smem_u32(&bar_w[ew][0]);
     auto w_bar = [&](uint32_t b) { return w_bar0 + b * 8u; };
     const bool upd = (p.kind == GEMM_FINAL && p.sink_mode == SINK_UPDATE_W);
@@ -564,13 +565,9 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
               add[q * 8 + 4] = bf16_lo(u.z); add[q * 8 + 5] = bf16_hi(u.z);
               add[q * 8 + 6] = bf16_lo(u.w); add[q * 8 + 7] = bf16_hi(u.w);
             }
-            if (p.kind == GEMM_POLY) {
+            const int dcol = gi - (gj0 + h * 32);        // this lane's diagonal element, if it is in the block
 #pragma unroll
-              for (int e = 0; e < 32; ++e) f[e] = fmaf(p.c, f[e], p.b * add[e]);
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) f[e] = sc * fmaf(p.a, add[e], f[e]);
-            }
+            for (int e = 0; e < 32; ++e) f[e] = fmaf(p.c, f[e], p.b * add[e]) + ((e == dcol) ? p.a : 0.0f);
           } else {
 #pragma unroll
             for (int e = 0; e < 32; ++e) f[e] *= sc;
@@ -945,7 +942,7 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int kind, int n_mats, in
   m = Maps5{&pl->b_k, &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin], &pl->b_mn};
   if (kind == GEMM_APPLY)
     return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
-  return pl->cg == 2 ? launch_one<2, true, 4>(st, m, p, pl->n_sms) : launch_one<1, true, 4>(st, m, p, pl->n_sms);
+  return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
 }
 
 }  // namespace muloco
