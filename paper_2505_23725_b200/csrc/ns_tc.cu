@@ -34,6 +34,7 @@
 // roles leave their loops, and the CTA frees its tensor memory and returns.
 #include <cuda.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <vector>
@@ -73,6 +74,8 @@ struct TcParams {
   int sink_mode;
   int a_tri, b_tri;           // left / right operand is a symmetric matrix of which only the tiles on
                               // or above the diagonal are stored
+  int b_wide, s_wide;         // tmB (MN-major right operand) / tmS (mirror-image boxes) is the 4-D form:
+                              // one copy brings both 64-column atoms (128 operand rows x 64 k) of a slab
   int64_t s, l;
   int* status;
 };
@@ -154,6 +157,21 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// 4-D forms for the maps that deliver two 64-column atoms of an MN-major operand in one copy
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
@@ -364,23 +382,23 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             if (CG == 1) tma_load_3d(dst, map, bar, c0, c1, mat);
             else tma_load_3d_pair(dst, map, bar, c0, c1, mat);
           };
-          const int k0 = kb * BK;
-          if (kb >= ka_mn) {
-            load(sa, &tmA, k0, a_row);
-          } else {
-            load(sa, &tmS, a_row, k0);
-            load(sa + BK * 128, &tmS, a_row + 64, k0);
-          }
-          if (!same) {
-            if (B_MN) {
-              load(sb, &tmB, b_off, k0);
-              load(sb + BK * 128, &tmB, b_off + 64, k0);
-            } else if (kb >= kb_mn) {
-              load(sb, &tmB, k0, b_off);
+          // an MN-major slab = two 64-column atoms of 64 k rows: one 4-D copy, or two 64 x 64 boxes
+          auto load_mn = [&](uint32_t dst, const CUtensorMap* map, bool wide, int col0, int k) {
+            if (wide) {
+              if (CG == 1) tma_load_4d(dst, map, bar, 0, k, col0 >> 6, mat);
+              else tma_load_4d_pair(dst, map, bar, 0, k, col0 >> 6, mat);
             } else {
-              load(sb, &tmS, b_off, k0);
-              load(sb + BK * 128, &tmS, b_off + 64, k0);
+              load(dst, map, col0, k);
+              load(dst + BK * 128, map, col0 + 64, k);
             }
+          };
+          const int k0 = kb * BK;
+          if (kb >= ka_mn) load(sa, &tmA, k0, a_row);
+          else load_mn(sa, &tmS, p.s_wide != 0, a_row, k0);
+          if (!same) {
+            if (B_MN) load_mn(sb, &tmB, p.b_wide != 0, b_off, k0);
+            else if (kb >= kb_mn) load(sb, &tmB, k0, b_off);
+            else load_mn(sb, &tmS, p.s_wide != 0, b_off, k0);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -758,6 +776,22 @@ bool encode_map(CUtensorMap* out, void* base, int64_t cols, int64_t rows, int64_
   return r == CUDA_SUCCESS;
 }
 
+// 4-D map over the same array for MN-major operands: [n_slots][cols/64][rows][64], box 64 x 64 x 2 x 1,
+// i.e. two consecutive 64-column atoms (64 rows of 128 bytes each, 8 KB apart in shared memory) per copy.
+// Needs cols % 64 == 0.
+bool encode_map_mn2(CUtensorMap* out, void* base, int64_t cols, int64_t rows, int64_t n_slots, int64_t ld) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn || (cols & 63) != 0) return false;
+  cuuint64_t dims[4] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64), (cuuint64_t)n_slots};
+  cuuint64_t strides[3] = {(cuuint64_t)ld * 2, 128, (cuuint64_t)rows * (cuuint64_t)ld * 2};
+  cuuint32_t box[4] = {64, (cuuint32_t)BK, 2, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool tc_encode_w_map(void* out_host, void* base, int64_t rows, int64_t cols, int transposed) {
@@ -846,6 +880,10 @@ struct TcGroupPlan {
   // operand of the apply, A and B for the blocks read from their mirror image); io: 64 x 32 boxes
   // for addend loads and result stores
   CUtensorMap x_k[2], x_mn[2], x_io[2], a_k, a_mn, a_io, b_k, b_mn, b_io;
+  // 4-D forms of the mn maps (both atoms of a slab in one copy); used when the column count is a
+  // multiple of 64 and the driver accepts the layout
+  CUtensorMap x_mn2[2], a_mn2, b_mn2;
+  bool wide_x = false, wide_s = false;
   int2* tiles_sym = nullptr;
   int n_tiles_sym = 0;
   int2* tiles_full = nullptr;
@@ -881,6 +919,12 @@ TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1,
   ok = ok && encode_map(&pl->b_k, B, s, s, chunk, lds, BK, 128, true);
   ok = ok && encode_map(&pl->b_io, B, s, s, chunk, lds, 64, 32, true);
   ok = ok && encode_map(&pl->b_mn, B, s, s, chunk, lds, 64, BK, true);
+  pl->wide_x = encode_map_mn2(&pl->x_mn2[0], pl->X[0], l, s, chunk, ldx) &&
+               encode_map_mn2(&pl->x_mn2[1], pl->X[1], l, s, chunk, ldx);
+  pl->wide_s = encode_map_mn2(&pl->a_mn2, A, s, s, chunk, lds) && encode_map_mn2(&pl->b_mn2, B, s, s, chunk, lds);
+  if (getenv("MULOCO_VERBOSE"))
+    fprintf(stderr, "muloco: Newton-Schulz plan %lld x %lld, chunk %d: one-copy MN-major slabs for X %s, for A/B %s\n",
+            (long long)s, (long long)l, chunk, pl->wide_x ? "yes" : "no", pl->wide_s ? "yes" : "no");
   if (!ok) {
     snprintf(err, errlen, "cuTensorMapEncodeTiled failed for shape %lld x %lld", (long long)s, (long long)l);
     delete pl;
@@ -933,13 +977,16 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int kind, int n_mats, in
   if (kind == GEMM_POLY) {
     p.N = (int)pl->s; p.Kd = (int)pl->s; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
     p.a_tri = 1; p.b_tri = 1;
-    m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, &pl->a_mn};
+    p.s_wide = pl->wide_s;
+    m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, pl->wide_s ? &pl->a_mn2 : &pl->a_mn};
     return pl->cg == 2 ? launch_one<2, false, 5>(st, m, p, pl->n_sms) : launch_one<1, false, 5>(st, m, p, pl->n_sms);
   }
   p.N = (int)pl->l; p.Kd = (int)pl->s; p.tiles = pl->tiles_full; p.n_tiles_per_mat = pl->n_tiles_full;
   // FINAL stores nothing through tmD; the map still has to be a valid one
   p.a_tri = 1;      // the left operand is the polynomial B, stored on and above the diagonal
-  m = Maps5{&pl->b_k, &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin], &pl->b_mn};
+  p.b_wide = pl->wide_x; p.s_wide = pl->wide_s;
+  m = Maps5{&pl->b_k, pl->wide_x ? &pl->x_mn2[xin] : &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin],
+            pl->wide_s ? &pl->b_mn2 : &pl->b_mn};
   if (kind == GEMM_APPLY)
     return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
   return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
