@@ -33,10 +33,10 @@ UNIT = "param-updates/s"
 
 # DRAM traffic of the Newton-Schulz GEMM launches per hidden-matrix parameter, worker and inner
 # step, from the ncu capture summarised in profiles/ns_tc_kernel_muon-only_K16_L2_d1024_F2816.md
-# (19.84 GB over the 30 launches of a 2-layer, K=16 inner step with 25,690,112 parameters per
+# (19.91 GB over the 30 launches of a 2-layer, K=16 inner step with 25,690,112 parameters per
 # replica).  It grows in proportion to the number of matrices, so it is scaled by the parameter
 # count; it holds for the d=1024, F=2816 shape mix only.
-NS_TRAFFIC_BYTES_PER_PARAM = {}   # empty while the kernel is newer than the capture: traffic is then reported as null
+NS_TRAFFIC_BYTES_PER_PARAM = {(1024, 2816): 19.909e9 / (25690112 * 16)}
 
 
 def load_peaks():
