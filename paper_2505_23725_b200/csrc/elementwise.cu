@@ -46,7 +46,8 @@ __global__ void __launch_bounds__(PRO_THREADS)
 prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_mode, int g_is_bf16,
                 float beta, int nesterov, XT* __restrict__ X, int64_t ldx, float* __restrict__ partials,
                 int tiles_j, int n_part) {
-  __shared__ float tile[PRO_TJ][PRO_TI + 1];
+  __shared__ float tile_raw[64 * 129];          // viewed as 128 x 33, 64 x 65 or 64 x 129 by the paths below
+  float (*tile)[PRO_TI + 1] = reinterpret_cast<float (*)[PRO_TI + 1]>(tile_raw);
   __shared__ float red[PRO_THREADS / 32];
   const int mat = blockIdx.y;
   const MatDesc d = mats[mat];
@@ -57,17 +58,27 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   // and the CTAs a tensor does not need write a zero partial sum.
   const bool pair_ok = ((((uintptr_t)d.m) & 7) == 0) &&
                        ((((uintptr_t)d.g) & ((src_mode == SRC_RAW_BF16 || (src_mode == SRC_MUON && g_is_bf16)) ? 3 : 7)) == 0);
-  const bool t64 = d.transposed && ((s & 1) == 0) && pair_ok;
-  const int tiles_i = t64 ? (int)((s + 63) / 64) : (int)((s + PRO_TI - 1) / PRO_TI);
-  const int tiles_jj = t64 ? (int)((l + 63) / 64) : tiles_j;
+  const bool src_is_bf16 = (src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16);
+  // tall tensors with a bf16 source: 128 x 64 tiles, four consecutive i per lane (8-byte pieces of the
+  // 2-byte stream, 256 bytes per warp and tensor row; the 64 x 64 path would read it in 128-byte pieces)
+  const bool t128 = d.transposed && src_is_bf16 && ((s & 3) == 0) && ((((uintptr_t)d.g) & 7) == 0) &&
+                    ((((uintptr_t)d.m) & 15) == 0);
+  const bool t64 = !t128 && d.transposed && ((s & 1) == 0) && pair_ok;
+  XT* Xm = X + (int64_t)mat * s * ldx;
+  // bf16 sources of tensors stored s x l: 32 x 256 tiles, eight consecutive j per thread, so that the
+  // 2-byte stream is read in 512-byte pieces per tile row like the 4-byte streams of the other paths
+  const bool vec8 = !d.transposed && src_is_bf16 && sizeof(XT) == 2 && ((l & 7) == 0) && ((ldx & 7) == 0) &&
+                    ((((uintptr_t)d.g | (uintptr_t)d.m | (uintptr_t)Xm) & 15) == 0);
+  const int tiles_i = t128 ? (int)((s + 127) / 128) : (t64 ? (int)((s + 63) / 64) : (int)((s + PRO_TI - 1) / PRO_TI));
+  const int tiles_jj = (t64 || t128) ? (int)((l + 63) / 64) : (vec8 ? (int)((l + 255) / 256) : tiles_j);
   if ((int)blockIdx.x >= tiles_i * tiles_jj) {
     if (threadIdx.x == 0) partials[(int64_t)mat * n_part + blockIdx.x] = 0.f;
     return;
   }
   const int ti = d.transposed ? (int)(blockIdx.x % tiles_i) : (int)(blockIdx.x / tiles_jj);
   const int tj = d.transposed ? (int)(blockIdx.x / tiles_i) : (int)(blockIdx.x % tiles_jj);
-  const int64_t i0 = (int64_t)ti * (t64 ? 64 : PRO_TI), j0 = (int64_t)tj * (t64 ? 64 : PRO_TJ);
-  XT* Xm = X + (int64_t)mat * s * ldx;
+  const int64_t i0 = (int64_t)ti * (t128 ? 128 : (t64 ? 64 : PRO_TI));
+  const int64_t j0 = (int64_t)tj * ((t64 || t128) ? 64 : (vec8 ? 256 : PRO_TJ));
   float ss = 0.f;
   const int tid = threadIdx.x;
 
@@ -86,7 +97,70 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
     return u;
   };
 
-  if (t64) {
+  if (t128) {
+    // tensor is l x s with a bf16 source: read rows j (128 consecutive i, four per lane), turn the tile
+    // through shared memory, write rows i of X (64 consecutive j per warp)
+    float (*t12)[129] = reinterpret_cast<float (*)[129]>(tile_raw);
+    const int lane = tid & 31, w = tid >> 5;
+    const int64_t i = i0 + 4 * lane;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {          // four rows at a time: their loads before their stores
+      uint2 graw[4];
+      float4 mv[4];
+      bool ok[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int64_t j = j0 + w + 8 * (half * 4 + r);
+        ok[r] = (j < l) && (i < s);
+        graw[r] = make_uint2(0u, 0u);
+        mv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!ok[r]) continue;
+        const int64_t idx = j * s + i;
+        graw[r] = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(d.g) + idx));
+        if (src_mode == SRC_MUON) mv[r] = *reinterpret_cast<const float4*>(d.m + idx);
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int jj = w + 8 * (half * 4 + r);
+        float u[4] = {0.f, 0.f, 0.f, 0.f};
+        if (ok[r]) {
+          const float g[4] = {__uint_as_float(graw[r].x << 16), __uint_as_float(graw[r].x & 0xFFFF0000u),
+                              __uint_as_float(graw[r].y << 16), __uint_as_float(graw[r].y & 0xFFFF0000u)};
+          if (src_mode == SRC_MUON) {
+            const float mold[4] = {mv[r].x, mv[r].y, mv[r].z, mv[r].w};
+            float mn[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              mn[e] = fmaf(beta, mold[e], g[e]);
+              u[e] = nesterov ? fmaf(beta, mn[e], g[e]) : mn[e];
+            }
+            *reinterpret_cast<float4*>(d.m + (j0 + jj) * s + i) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) u[e] = g[e];
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) ss = fmaf(u[e], u[e], ss);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) t12[jj][4 * lane + e] = u[e];
+      }
+    }
+    __syncthreads();
+    const int64_t j = j0 + 2 * lane;
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+      const int ii = w + 8 * r;
+      const int64_t ix = i0 + ii;
+      if (ix >= s || j >= l) continue;
+      const float a0 = t12[2 * lane][ii], a1 = t12[2 * lane + 1][ii];
+      if (j + 1 < l) {
+        store_x2(Xm + ix * ldx + j, a0, a1);
+      } else {
+        Xm[ix * ldx + j] = to_x<XT>(a0);
+      }
+    }
+  } else if (t64) {
     // tensor is l x s: read rows j (64 consecutive i = 256 bytes per warp, two per lane), turn the
     // tile through shared memory, write rows i of X (64 consecutive j per warp)
     float (*t6)[65] = reinterpret_cast<float (*)[65]>(&tile[0][0]);
@@ -152,8 +226,64 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   }
   const bool vec4 = !d.transposed && ((l & 3) == 0) && ((ldx & 3) == 0) &&
                     ((((uintptr_t)d.g | (uintptr_t)d.m) & 15) == 0) && ((((uintptr_t)Xm) & 15) == 0);
-  if (t64) {
+  if (t64 || t128) {
     // handled above
+  } else if (vec8) {
+    const int tx = tid & 31, ty = tid >> 5;   // 32 lanes x 8 columns, 8 warps x 4 rows
+    const int64_t j = j0 + tx * 8;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {    // two rows at a time: all loads of both rows before their stores
+      uint4 graw[2];
+      float4 mo[2][2];
+      bool ok[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int64_t i = i0 + ty + (half * 2 + r) * 8;
+        ok[r] = (i < s) && (j < l);
+        graw[r] = make_uint4(0u, 0u, 0u, 0u);
+        mo[r][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        mo[r][1] = mo[r][0];
+        if (!ok[r]) continue;
+        const int64_t idx = i * l + j;
+        graw[r] = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(d.g) + idx));
+        if (src_mode == SRC_MUON) {
+          mo[r][0] = *reinterpret_cast<const float4*>(d.m + idx);
+          mo[r][1] = *reinterpret_cast<const float4*>(d.m + idx + 4);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        if (!ok[r]) continue;
+        const int64_t i = i0 + ty + (half * 2 + r) * 8;
+        const int64_t idx = i * l + j;
+        const uint32_t w[4] = {graw[r].x, graw[r].y, graw[r].z, graw[r].w};
+        float g[8], u[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          g[2 * q] = __uint_as_float(w[q] << 16);
+          g[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+        }
+        if (src_mode == SRC_MUON) {
+          const float mold[8] = {mo[r][0].x, mo[r][0].y, mo[r][0].z, mo[r][0].w,
+                                 mo[r][1].x, mo[r][1].y, mo[r][1].z, mo[r][1].w};
+          float mn[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            mn[e] = fmaf(beta, mold[e], g[e]);
+            u[e] = nesterov ? fmaf(beta, mn[e], g[e]) : mn[e];
+          }
+          *reinterpret_cast<float4*>(d.m + idx) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+          *reinterpret_cast<float4*>(d.m + idx + 4) = make_float4(mn[4], mn[5], mn[6], mn[7]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) u[e] = g[e];
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss = fmaf(u[e], u[e], ss);
+        store_x4(Xm + i * ldx + j, make_float4(u[0], u[1], u[2], u[3]));
+        store_x4(Xm + i * ldx + j + 4, make_float4(u[4], u[5], u[6], u[7]));
+      }
+    }
   } else if (vec4) {
     // tensor is s x l with 16-byte aligned rows: four consecutive j per thread.  All loads of
     // the thread's four rows are issued before the first store (the stores to m would
