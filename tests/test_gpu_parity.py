@@ -568,3 +568,53 @@ def test_nonfinite_gradient_of_a_hidden_matrix_is_reported():
     assert e.value.status == binding.ENONFINITE
     gpu.sync_status()                                   # the flag is cleared once read
     gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# bf16 sources: every access shape of the staging kernel (wide and tall tensors, aligned and not)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("m,n", [(384, 256), (96, 1032), (96, 1031), (130, 96), (257, 131), (132, 514), (1024, 64),
+                                 (64, 1024), (8, 24), (24, 8)])
+def test_newton_schulz_bf16_input_shapes(ns_ctx, m, n):
+    import torch
+    rng = np.random.default_rng(1000 + 3 * m + n)
+    X = torch.from_numpy(synth.lowrank_plus_noise(rng, m, n)).cuda().to(torch.bfloat16)
+    ref = O.newton_schulz(_np(X.float()))
+    for mode, tol in (("fp32", 1e-4), ("bf16", 2e-2)):
+        out = ns_ctx.newton_schulz(X, out_dtype=torch.float32, ns_mode=mode)
+        assert relfro(_np(out), ref) < tol, f"{mode} {m}x{n}: {relfro(_np(out), ref):.3e}"
+    ns_ctx.sync_status()
+
+
+@pytest.mark.parametrize("d,F", [(64, 96), (96, 200), (68, 130)])
+def test_inner_steps_with_bf16_gradients(d, F):
+    # momentum (fp32, 1e-6) and the Muon update (2e-2 relative Frobenius in the bf16 engine) with
+    # bf16 gradients; the oracle gets the same bf16-rounded values
+    import dataclasses
+    import torch
+    w = dataclasses.replace(configs.mini_workload(K=2, H=2, L=1, d=d, F=F, vocab=40, norms=True, ns_mode="bf16"),
+                            grad_dtype="bf16")
+    rng = np.random.default_rng(d + F)
+    init = synth.init_weights(rng, w.tensors)
+    gpu = gpu_for(w, init)
+    orc = oracle_for(w, init)
+    for step in range(2):
+        gs = [synth.host_gradients(rng, w.tensors) for _ in range(w.K)]
+        gb = [[torch.from_numpy(np.ascontiguousarray(g)).cuda().to(torch.bfloat16) for g in gk] for gk in gs]
+        before = [[_np(gpu.theta_k[k][i]).copy() for i in range(gpu.n)] for k in range(w.K)]
+        gpu.inner_step(-1, gb)
+        gpu.sync_status()
+        for k in range(w.K):
+            for i in range(gpu.n):
+                orc.theta_k[k][i][...] = before[k][i]
+        orc.inner_step_all([[_np(g.float()) for g in gk] for gk in gb])
+        for k in range(w.K):
+            for i, t in enumerate(w.tensors):
+                assert_close_1e6(_np(gpu.state1[k][i]), orc.state1[k][i], f"state1 k={k} {t.name} step {step}")
+                if t.kind == configs.MUON:
+                    upd, ref = _np(gpu.theta_k[k][i]).astype(np.float64) - before[k][i], \
+                        orc.theta_k[k][i].astype(np.float64) - before[k][i]
+                    assert relfro(upd, ref) < 2e-2, f"Muon update k={k} {t.name} step {step}: {relfro(upd, ref):.3e}"
+                else:
+                    assert_close_1e6(_np(gpu.theta_k[k][i]), orc.theta_k[k][i], f"theta k={k} {t.name} step {step}")
+    gpu.close()
