@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(PRO_THREADS)
 prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_mode, int g_is_bf16,
                 float beta, int nesterov, XT* __restrict__ X, int64_t ldx, float* __restrict__ partials,
                 int tiles_j, int n_part) {
-  __shared__ float tile_raw[64 * 129];          // viewed as 128 x 33, 64 x 65 or 64 x 129 by the paths below
+  __shared__ float tile_raw[PRO_TJ * (PRO_TI + 1)];   // viewed as 128 x 33 or 64 x 65 floats, or 64 x 130 bf16
   float (*tile)[PRO_TI + 1] = reinterpret_cast<float (*)[PRO_TI + 1]>(tile_raw);
   __shared__ float red[PRO_THREADS / 32];
   const int mat = blockIdx.y;
@@ -61,8 +61,8 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   const bool src_is_bf16 = (src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16);
   // tall tensors with a bf16 source: 128 x 64 tiles, four consecutive i per lane (8-byte pieces of the
   // 2-byte stream, 256 bytes per warp and tensor row; the 64 x 64 path would read it in 128-byte pieces)
-  const bool t128 = d.transposed && src_is_bf16 && ((s & 3) == 0) && ((((uintptr_t)d.g) & 7) == 0) &&
-                    ((((uintptr_t)d.m) & 15) == 0);
+  const bool t128 = d.transposed && src_is_bf16 && sizeof(XT) == 2 && ((s & 3) == 0) &&
+                    ((((uintptr_t)d.g) & 7) == 0) && ((((uintptr_t)d.m) & 15) == 0);
   const bool t64 = !t128 && d.transposed && ((s & 1) == 0) && pair_ok;
   XT* Xm = X + (int64_t)mat * s * ldx;
   // bf16 sources of tensors stored s x l: 32 x 256 tiles, eight consecutive j per thread, so that the
@@ -99,8 +99,10 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
 
   if (t128) {
     // tensor is l x s with a bf16 source: read rows j (128 consecutive i, four per lane), turn the tile
-    // through shared memory, write rows i of X (64 consecutive j per warp)
-    float (*t12)[129] = reinterpret_cast<float (*)[129]>(tile_raw);
+    // through shared memory (already rounded to bf16, which is what X holds), write rows i of X
+    // (64 consecutive j per warp)
+    __nv_bfloat16 (*t12)[130] = reinterpret_cast<__nv_bfloat16 (*)[130]>(tile_raw);
+    static_assert(64 * 130 * 2 <= PRO_TJ * (PRO_TI + 1) * 4, "staging tile");
     const int lane = tid & 31, w = tid >> 5;
     const int64_t i = i0 + 4 * lane;
 #pragma unroll
@@ -143,7 +145,7 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
           for (int e = 0; e < 4; ++e) ss = fmaf(u[e], u[e], ss);
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) t12[jj][4 * lane + e] = u[e];
+        for (int e = 0; e < 4; ++e) t12[jj][4 * lane + e] = __float2bfloat16_rn(u[e]);
       }
     }
     __syncthreads();
@@ -153,11 +155,13 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
       const int ii = w + 8 * r;
       const int64_t ix = i0 + ii;
       if (ix >= s || j >= l) continue;
-      const float a0 = t12[2 * lane][ii], a1 = t12[2 * lane + 1][ii];
-      if (j + 1 < l) {
-        store_x2(Xm + ix * ldx + j, a0, a1);
-      } else {
-        Xm[ix * ldx + j] = to_x<XT>(a0);
+      if constexpr (sizeof(XT) == 2) {
+        const __nv_bfloat16 a0 = t12[2 * lane][ii], a1 = t12[2 * lane + 1][ii];
+        if (j + 1 < l) {
+          *reinterpret_cast<__nv_bfloat162*>(Xm + ix * ldx + j) = __halves2bfloat162(a0, a1);
+        } else {
+          Xm[ix * ldx + j] = a0;
+        }
       }
     }
   } else if (t64) {
