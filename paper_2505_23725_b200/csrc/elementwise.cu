@@ -41,7 +41,9 @@ __device__ __forceinline__ void store_x4(__nv_bfloat16* p, float4 u) {
 
 // One CTA = one 32 x 128 tile of X (s x l view) of one matrix.
 // The value that enters the sum of squares is the fp32 U (before bf16 rounding).
-template <typename XT>
+// BF16SRC: the source (gradient, or the standalone call's input) is bf16; only that instantiation
+// carries the bf16 access shapes, so the fp32-source kernel keeps its register count.
+template <typename XT, bool BF16SRC>
 __global__ void __launch_bounds__(PRO_THREADS)
 prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_mode, int g_is_bf16,
                 float beta, int nesterov, XT* __restrict__ X, int64_t ldx, float* __restrict__ partials,
@@ -58,16 +60,16 @@ prologue_kernel(const MatDesc* __restrict__ mats, int64_t s, int64_t l, int src_
   // and the CTAs a tensor does not need write a zero partial sum.
   const bool pair_ok = ((((uintptr_t)d.m) & 7) == 0) &&
                        ((((uintptr_t)d.g) & ((src_mode == SRC_RAW_BF16 || (src_mode == SRC_MUON && g_is_bf16)) ? 3 : 7)) == 0);
-  const bool src_is_bf16 = (src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16);
+  const bool src_is_bf16 = BF16SRC && ((src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16));
   // tall tensors with a bf16 source: 128 x 64 tiles, four consecutive i per lane (8-byte pieces of the
   // 2-byte stream, 256 bytes per warp and tensor row; the 64 x 64 path would read it in 128-byte pieces)
-  const bool t128 = d.transposed && src_is_bf16 && sizeof(XT) == 2 && ((s & 3) == 0) &&
+  const bool t128 = BF16SRC && d.transposed && src_is_bf16 && sizeof(XT) == 2 && ((s & 3) == 0) &&
                     ((((uintptr_t)d.g) & 7) == 0) && ((((uintptr_t)d.m) & 15) == 0);
   const bool t64 = !t128 && d.transposed && ((s & 1) == 0) && pair_ok;
   XT* Xm = X + (int64_t)mat * s * ldx;
   // bf16 sources of tensors stored s x l: 32 x 256 tiles, eight consecutive j per thread, so that the
   // 2-byte stream is read in 512-byte pieces per tile row like the 4-byte streams of the other paths
-  const bool vec8 = !d.transposed && src_is_bf16 && sizeof(XT) == 2 && ((l & 7) == 0) && ((ldx & 7) == 0) &&
+  const bool vec8 = BF16SRC && !d.transposed && src_is_bf16 && sizeof(XT) == 2 && ((l & 7) == 0) && ((ldx & 7) == 0) &&
                     ((((uintptr_t)d.g | (uintptr_t)d.m | (uintptr_t)Xm) & 15) == 0);
   const int tiles_i = t128 ? (int)((s + 127) / 128) : (t64 ? (int)((s + 63) / 64) : (int)((s + PRO_TI - 1) / PRO_TI));
   const int tiles_jj = (t64 || t128) ? (int)((l + 63) / 64) : (vec8 ? (int)((l + 255) / 256) : tiles_j);
@@ -535,13 +537,19 @@ void launch_prologue(cudaStream_t st, const MatDesc* mats, int n_mats, int64_t s
   for (int m0 = 0; m0 < n_mats; m0 += 65535) {
     const int nm = (n_mats - m0 < 65535) ? (n_mats - m0) : 65535;
     dim3 grid((unsigned)n_part, (unsigned)nm);
+    const bool bf16_src = (src_mode == SRC_RAW_BF16) || (src_mode == SRC_MUON && g_is_bf16);
     if (x_is_f32)
-      prologue_kernel<float><<<grid, PRO_THREADS, 0, st>>>(
+      prologue_kernel<float, false><<<grid, PRO_THREADS, 0, st>>>(
           mats + m0, s, l, src_mode, g_is_bf16, beta, nesterov,
           reinterpret_cast<float*>(X) + (int64_t)m0 * s * ldx, ldx, partials + (int64_t)m0 * n_part,
           tiles_j, n_part);
+    else if (bf16_src)
+      prologue_kernel<__nv_bfloat16, true><<<grid, PRO_THREADS, 0, st>>>(
+          mats + m0, s, l, src_mode, g_is_bf16, beta, nesterov,
+          reinterpret_cast<__nv_bfloat16*>(X) + (int64_t)m0 * s * ldx, ldx,
+          partials + (int64_t)m0 * n_part, tiles_j, n_part);
     else
-      prologue_kernel<__nv_bfloat16><<<grid, PRO_THREADS, 0, st>>>(
+      prologue_kernel<__nv_bfloat16, false><<<grid, PRO_THREADS, 0, st>>>(
           mats + m0, s, l, src_mode, g_is_bf16, beta, nesterov,
           reinterpret_cast<__nv_bfloat16*>(X) + (int64_t)m0 * s * ldx, ldx,
           partials + (int64_t)m0 * n_part, tiles_j, n_part);
