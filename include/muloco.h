@@ -48,8 +48,9 @@ typedef enum {
   MULOCO_ESHAPE = 2,     /* unsupported shape */
   MULOCO_ENOMEM = 3,     /* workspace allocation failed */
   MULOCO_ECUDA = 4,      /* CUDA runtime/driver error, or no device */
-  MULOCO_ENONFINITE = 5, /* device saw a non-finite pseudogradient, or a non-finite gradient /
-                            momentum of a hidden matrix (its Frobenius norm)          */
+  MULOCO_ENONFINITE = 5, /* device saw a non-finite pseudogradient, a non-finite gradient /
+                            momentum of a hidden matrix (its Frobenius norm), or a
+                            non-finite gradient of an AdamW tensor                    */
   MULOCO_ETIMEOUT = 6,   /* a bounded wait inside a kernel ran out */
   MULOCO_ESTATE = 7      /* call order / state blob mismatch */
 } muloco_status;
@@ -192,7 +193,12 @@ MULOCO_API int32_t muloco_fragments_due(const muloco_ctx* ctx, int64_t step, int
  * O has the same shape (o_dtype).  Each matrix is divided by its Frobenius norm
  * (+ ns_eps) first; matrices with rows > cols are iterated on their transpose.
  * ns_mode MULOCO_NS_BF16 runs the tensor-core engine (bf16 operands, fp32
- * accumulation), MULOCO_NS_FP32 the fp32 engine.  X and O must not overlap. */
+ * accumulation), MULOCO_NS_FP32 the fp32 engine.  X and O must not overlap.
+ * Accuracy against the iteration in exact arithmetic (relative Frobenius error):
+ * 1e-4 for the fp32 engine, 2e-2 for the bf16 engine.  The bf16 engine holds its
+ * bound only from min(rows, cols) = 64 on; matrices with a smaller min-dimension
+ * (also inside muloco_inner_step) are always served by the fp32 engine, whatever
+ * mode is asked, and meet the fp32 bound. */
 MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* ctx, const void* X, int32_t x_dtype, void* O,
                                    int32_t o_dtype, int32_t batch, int64_t rows, int64_t cols,
                                    int32_t ns_mode);
@@ -220,7 +226,12 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* ctx, const void* X, in
  * MULOCO_ESHAPE and explains the sizes in errbuf -- use muloco_newton_schulz then.
  * errbuf (host, may be NULL) receives a NUL-terminated message on failure.
  * The work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default stream) of
- * the CURRENT device.
+ * the CURRENT device; the call copies nothing from host memory (its small tables are
+ * written by a kernel from the arguments), so nothing on the host has to outlive it.
+ * Only argument and launch errors are reported: there is no context and no status
+ * word, so a NaN or Inf in X is not detected -- the matrix that holds it comes out
+ * non-finite and the call still returns MULOCO_OK (muloco_newton_schulz followed by
+ * muloco_sync_status reports MULOCO_ENONFINITE for the same input).
  *
  * The first call on each device resolves the scratch's device address (once per
  * device, that device being current); make that first call before starting any

@@ -110,17 +110,23 @@ def load_library():
     return lib
 
 
-def newton_schulz_static(X, stream=None):
+def newton_schulz_static(X, stream=None, out=None):
     """muloco_newton_schulz_static: fp32 Newton-Schulz of a small [batch, rows, cols]
-    (or [rows, cols]) float32 CUDA tensor without any device allocation by the library
-    (the output tensor is allocated here, by torch, before the call).  For callers that
-    may not allocate; sizes beyond the library's fixed scratch raise MulocoError(ESHAPE)."""
+    (or [rows, cols]) float32 CUDA tensor without any device allocation by the library.
+    The result goes to `out` (same shape, float32, contiguous) when given; otherwise the
+    output tensor is allocated here, by torch, before the call.  For callers that may
+    not allocate; sizes beyond the library's fixed scratch raise MulocoError(ESHAPE)."""
     import torch
     lib = load_library()
     x = (X if X.dim() == 3 else X.unsqueeze(0)).contiguous()
     if x.dtype != torch.float32 or not x.is_cuda:
         raise ValueError("expects a float32 CUDA tensor")
-    o = torch.empty_like(x)
+    if out is None:
+        o = torch.empty_like(x)
+    else:
+        o = out if out.dim() == 3 else out.unsqueeze(0)
+        if o.shape != x.shape or o.dtype != torch.float32 or not o.is_contiguous() or o.device != x.device:
+            raise ValueError("out must be a contiguous float32 tensor of X's shape on X's device")
     st = stream if stream is not None else torch.cuda.current_stream(x.device)
     err = C.create_string_buffer(256)
     with torch.cuda.device(x.device):

@@ -40,6 +40,7 @@ struct Group {
   int chunk = 0;
   int n_part = 0;
   int elt = 2;
+  int mode = MULOCO_NS_BF16;   // engine that serves this group (see engine_for)
   WsLayout ws;
   TcGroupPlan* plan = nullptr;
 };
@@ -66,6 +67,14 @@ constexpr int RING = 3;
 constexpr uint32_t STATE_MAGIC = 0x4d4c4331u;   // "MLC1"
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// The bf16 engine holds its 2e-2 tolerance from a min-dimension of 64 on (measured against the fp64
+// iteration: 1.0-1.5e-2 there, 1.9-3.8e-2 for 8..48 rows, where too few roundings average out), so
+// smaller matrices always take the fp32 engine; their cost is negligible.
+constexpr int64_t BF16_MIN_S = 64;
+int engine_for(int requested_mode, int64_t s) {
+  return (requested_mode == MULOCO_NS_BF16 && s >= BF16_MIN_S) ? MULOCO_NS_BF16 : MULOCO_NS_FP32;
+}
 
 WsLayout make_layout(int64_t s, int64_t ldx, int64_t lds, int chunk, int n_part, int elt) {
   WsLayout w;
@@ -233,6 +242,7 @@ void destroy_group(Group& g) {
 
 // Sets up a group's layout (and tensor-core plan in bf16 mode) inside workspace `ws`.
 muloco_status setup_group(muloco_ctx* c, Group& g, char* ws, int mode) {
+  g.mode = mode;
   g.elt = (mode == MULOCO_NS_BF16) ? 2 : 4;
   g.n_part = prologue_partials_per_matrix(g.s, g.l);
   g.ws = make_layout(g.s, g.ldx, g.lds, g.chunk, g.n_part, g.elt);
@@ -487,7 +497,6 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
     }
     c->groups[gidx[key]].tensors.push_back(i);
   }
-  const int elt = (cfg->ns_mode == MULOCO_NS_BF16) ? 2 : 4;
   // default budget: 6 GiB, less when the device is nearly full (the state of the largest
   // configurations leaves only a few GiB)
   size_t budget = cfg->workspace_bytes ? (size_t)cfg->workspace_bytes : ((size_t)6 << 30);
@@ -499,6 +508,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
   size_t need = 0;
   for (Group& g : c->groups) {
     const int np = prologue_partials_per_matrix(g.s, g.l);
+    const int elt = (engine_for(cfg->ns_mode, g.s) == MULOCO_NS_BF16) ? 2 : 4;
     const size_t per_slot = make_layout(g.s, g.ldx, g.lds, 1, np, elt).total;
     g.chunk = pick_chunk((int64_t)g.tensors.size() * K, per_slot, budget);
     need = std::max(need, make_layout(g.s, g.ldx, g.lds, g.chunk, np, elt).total);
@@ -512,7 +522,7 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
     c->ws_bytes = need;
   }
   for (Group& g : c->groups) {
-    muloco_status s = setup_group(c, g, c->ws, cfg->ns_mode);
+    muloco_status s = setup_group(c, g, c->ws, engine_for(cfg->ns_mode, g.s));
     if (s != MULOCO_OK) return bail(s);
   }
 
@@ -678,7 +688,7 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
     }
     for (int m0 = 0; m0 < count; m0 += g.chunk) {
       const int cnt = std::min(g.chunk, count - m0);
-      rs = run_ns_chunk(c, g, c->ws, c->d_mats + group_begin[gi] + m0, cnt, f.ns_mode, SRC_MUON,
+      rs = run_ns_chunk(c, g, c->ws, c->d_mats + group_begin[gi] + m0, cnt, g.mode, SRC_MUON,
                         SINK_UPDATE_W, g_is_bf16);
       if (rs != MULOCO_OK) return rs;
     }
@@ -695,7 +705,7 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
     }
     {
       PhaseTimer t(c, MULOCO_PH_ADAMW);
-      launch_adamw(c->st, c->d_adam, (int)na, units, g_is_bf16, f.adam_beta1, f.adam_beta2, f.adam_eps);
+      launch_adamw(c->st, c->d_adam, (int)na, units, g_is_bf16, f.adam_beta1, f.adam_beta2, f.adam_eps, c->d_status);
       c->launches += 1;
     }
     if (c->host_mode) {
@@ -848,6 +858,7 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* c, const void* X, int3
   if (batch == 0) return MULOCO_OK;
   const int64_t s = std::min(rows, cols), l = std::max(rows, cols);
   Group& g = c->sa_group;
+  ns_mode = engine_for(ns_mode, s);
   const int elt = (ns_mode == MULOCO_NS_BF16) ? 2 : 4;
   const int64_t ldx = (l + 7) / 8 * 8, lds = (s + 7) / 8 * 8;
   const int np = prologue_partials_per_matrix(s, l);
@@ -1027,7 +1038,7 @@ MULOCO_API muloco_status muloco_sync_status(muloco_ctx* c) {
   if (h & ST_TIMEOUT) return fail(c, MULOCO_ETIMEOUT, "a bounded wait inside a kernel ran out");
   if (h & ST_BOUNDS) return fail(c, MULOCO_ECUDA, "a kernel rejected an out-of-range index");
   if (h & ST_NONFINITE)
-    return fail(c, MULOCO_ENONFINITE, "non-finite value: a pseudogradient, or the Newton-Schulz input of a hidden matrix");
+    return fail(c, MULOCO_ENONFINITE, "non-finite value: a pseudogradient, the Newton-Schulz input of a hidden matrix, or a gradient given to AdamW");
   return MULOCO_OK;
 }
 

@@ -466,7 +466,11 @@ __device__ __forceinline__ void adam_elem(float g, float& m, float& v, float& th
 
 __global__ void __launch_bounds__(ADAM_THREADS)
 adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int g_is_bf16, float beta1,
-             float beta2, float eps) {
+             float beta2, float eps, int* __restrict__ status) {
+  // a gradient that is not finite would poison m, v and theta for good: it is flagged (the step is
+  // still applied, like every other kernel here: nothing aborts)
+  bool bad = false;
+  auto check = [&](float g) { bad |= !(fabsf(g) <= 3.402823466e38f); };
   for (int64_t unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
     const int si = find_adam_seg(segs, n_segs, unit);
     const AdamSeg s = segs[si];
@@ -496,6 +500,7 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
             g = __ldcs(g4 + i);
           }
           float4 m = m4[i], v = v4[i], t = t4[i];
+          check(g.x); check(g.y); check(g.z); check(g.w);
           adam_elem(g.x, m.x, v.x, t.x, beta1, beta2, eps, s);
           adam_elem(g.y, m.y, v.y, t.y, beta1, beta2, eps, s);
           adam_elem(g.z, m.z, v.z, t.z, beta1, beta2, eps, s);
@@ -506,6 +511,7 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
       for (int64_t i = (int64_t)n4 * 4 + threadIdx.x; i < cnt; i += ADAM_THREADS) {
         float g = load_g(s.g, base + i, g_is_bf16);
         float m = s.m[base + i], v = s.v[base + i], t = s.theta[base + i];
+        check(g);
         adam_elem(g, m, v, t, beta1, beta2, eps, s);
         s.m[base + i] = m; s.v[base + i] = v; s.theta[base + i] = t;
       }
@@ -513,11 +519,13 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
       for (int64_t i = threadIdx.x; i < cnt; i += ADAM_THREADS) {
         float g = load_g(s.g, base + i, g_is_bf16);
         float m = s.m[base + i], v = s.v[base + i], t = s.theta[base + i];
+        check(g);
         adam_elem(g, m, v, t, beta1, beta2, eps, s);
         s.m[base + i] = m; s.v[base + i] = v; s.theta[base + i] = t;
       }
     }
   }
+  if (status && __syncthreads_or(bad ? 1 : 0) && threadIdx.x == 0) atomicOr(status, ST_NONFINITE);
 }
 
 }  // namespace
@@ -565,12 +573,12 @@ void launch_finalize_scales(cudaStream_t st, const float* partials, int n_part, 
 }
 
 void launch_adamw(cudaStream_t st, const AdamSeg* segs, int n_segs, int64_t n_units, int g_is_bf16,
-                  float beta1, float beta2, float eps) {
+                  float beta1, float beta2, float eps, int* status) {
   if (n_units <= 0 || n_segs <= 0) return;
   // one unit per CTA, launched in address order (the resident CTAs then share DRAM pages)
   int64_t blocks = n_units < 0x7fffffffLL ? n_units : 0x7fffffffLL;
   adamw_kernel<<<(unsigned)blocks, ADAM_THREADS, 0, st>>>(segs, n_segs, n_units, g_is_bf16, beta1,
-                                                          beta2, eps);
+                                                          beta2, eps, status);
 }
 
 }  // namespace muloco

@@ -84,8 +84,9 @@ struct AdamSeg {
   float inv_sqrt_bc2;   // 1 / sqrt(1 - beta2^t)
 };
 constexpr int ADAM_UNIT = 2048;
+// status: device status word; a non-finite gradient raises ST_NONFINITE (NULL: not checked)
 void launch_adamw(cudaStream_t st, const AdamSeg* segs, int n_segs, int64_t n_units, int g_is_bf16,
-                  float beta1, float beta2, float eps);
+                  float beta1, float beta2, float eps, int* status);
 
 // Outer sync: one entry per tensor of the fragment.
 struct SyncSeg {

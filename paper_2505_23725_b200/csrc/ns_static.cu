@@ -1,7 +1,9 @@
 // muloco_newton_schulz_static: Newton-Schulz on a small batch with NO device
 // allocation.  Its scratch (staged X, Gram and polynomial matrices, norm partials,
-// descriptor table, status word) lives in one file-scope __device__ array of fixed
-// size, so the call never reaches cudaMalloc/cudaFree.  It is meant for callers that
+// descriptor table) lives in one file-scope __device__ array of fixed size, so the
+// call never reaches cudaMalloc/cudaFree.  The descriptor table is written by a
+// small kernel from by-value arguments, so the call reads no host memory after it
+// returns.  It is meant for callers that
 // must not allocate: code that runs after a framework's caching allocator has
 // reserved the whole device (a raw cudaMalloc there can fail or fragment the pool),
 // and latency-sensitive loops that cannot afford the device-wide synchronisation an
@@ -38,6 +40,24 @@ std::mutex g_setup_mutex;
 
 size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
+// One descriptor per matrix of the batch, written on the device: X and O are
+// [batch][rows][cols]; the standalone sink stores O and uses no optimizer fields.
+__global__ void static_descs_kernel(MatDesc* __restrict__ mats, const float* X, float* O, int batch,
+                                    int64_t numel, int transposed) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= batch) return;
+  MatDesc d;
+  d.g = X + (size_t)j * numel;
+  d.m = nullptr;
+  d.w = O + (size_t)j * numel;
+  d.lr_eff = 0.f;
+  d.wd_term = 0.f;
+  d.transposed = transposed;
+  d.pad = 0;
+  d.wmap = nullptr;
+  mats[j] = d;
+}
+
 muloco_status fail(char* errbuf, size_t errlen, muloco_status s, const char* fmt, long long a = 0,
                    long long b = 0, long long c = 0) {
   if (errbuf && errlen) snprintf(errbuf, errlen, fmt, a, b, c);
@@ -62,9 +82,8 @@ extern "C" MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, 
   const int64_t ldx = (l + 7) / 8 * 8, lds = (s + 7) / 8 * 8;
   const int n_part = prologue_partials_per_matrix(s, l);
 
-  // carve the scratch: status | descriptors | X0 | X1 | A | B | partials | scales
+  // carve the scratch: descriptors | X0 | X1 | A | B | partials | scales
   size_t off = 0;
-  const size_t o_status = off; off += 256;
   const size_t o_mats = off;   off += up256((size_t)batch * sizeof(MatDesc));
   const size_t xb = up256((size_t)batch * s * ldx * sizeof(float));
   const size_t sb = up256((size_t)batch * s * lds * sizeof(float));
@@ -99,23 +118,11 @@ extern "C" MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, 
   }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
 
-  MatDesc hm[kMaxBatch];
-  for (int j = 0; j < batch; ++j) {
-    hm[j].g = X + (size_t)j * rows * cols;
-    hm[j].m = nullptr;
-    hm[j].w = O + (size_t)j * rows * cols;
-    hm[j].lr_eff = 0.f; hm[j].wd_term = 0.f;
-    hm[j].transposed = rows > cols;
-    hm[j].pad = 0;
-    hm[j].wmap = nullptr;
-  }
+  // Every region of the scratch is fully written by this call before it is read (descriptors
+  // here, X0 and the partial sums by the prologue, the scales, A, B and X1 by the kernels that
+  // follow on the same stream), so nothing has to be cleared and nothing of an earlier call leaks in.
   MatDesc* d_mats = reinterpret_cast<MatDesc*>(base + o_mats);
-  int* d_status = reinterpret_cast<int*>(base + o_status);
-  // the status word must start at zero; everything else is fully written before it is read
-  e = cudaMemsetAsync(d_status, 0, sizeof(int), st);
-  if (e == cudaSuccess)   // pageable source: staged before the call returns, so hm may go out of scope
-    e = cudaMemcpyAsync(d_mats, hm, (size_t)batch * sizeof(MatDesc), cudaMemcpyHostToDevice, st);
-  if (e != cudaSuccess) return fail(errbuf, errbuf_len, MULOCO_ECUDA, "table upload failed (error %lld)", (long long)e);
+  static_descs_kernel<<<1, kMaxBatch, 0, st>>>(d_mats, X, O, batch, rows * cols, rows > cols ? 1 : 0);
 
   float* X0 = reinterpret_cast<float*>(base + o_x0);
   float* X1 = reinterpret_cast<float*>(base + o_x1);
@@ -124,10 +131,10 @@ extern "C" MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, 
   float* partials = reinterpret_cast<float*>(base + o_part);
   float2* scales = reinterpret_cast<float2*>(base + o_scales);
   launch_prologue(st, d_mats, batch, s, l, SRC_RAW_F32, 0, 0.f, 0, X0, 1, ldx, partials);
-  launch_finalize_scales(st, partials, n_part, batch, 1e-7f, scales);
+  launch_finalize_scales(st, partials, n_part, batch, 1e-7f, scales);   // no status word: see the header
   NsIterArgs a;
   a.a = 3.4445f; a.b = -4.7750f; a.c = 2.0315f;   // Section 2, "Muon"
-  a.mats = d_mats; a.sink_mode = SINK_STORE_F32; a.status = d_status;
+  a.mats = d_mats; a.sink_mode = SINK_STORE_F32; a.status = nullptr;
   float* Xb[2] = {X0, X1};
   for (int it = 0; it < 5; ++it) {
     float* Xin = Xb[it & 1];
