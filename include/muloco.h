@@ -283,6 +283,22 @@ MULOCO_API muloco_status muloco_set_timing(muloco_ctx* ctx, int32_t enabled);
  * last call to *launches (either may be NULL), then resets both. */
 MULOCO_API muloco_status muloco_get_timings(muloco_ctx* ctx, float* ms, int64_t* launches);
 
+/* Test hooks for the failure path of the tensor-core Newton-Schulz kernel, whose every
+ * device-side wait (on a copy, on the tensor cores, on another CTA's tiles) has a time limit.
+ *   MULOCO_DEBUG_WAIT_LIMIT_NS : that limit in nanoseconds (0 restores the default of 2 s).
+ *   MULOCO_DEBUG_WITHHOLD_COPY : value != 0 makes the NEXT tensor-core launch of this context
+ *       leave out one operand copy of its first tile, so that the waits for it run out: the
+ *       kernel gives up cleanly (every CTA frees its tensor memory and returns) and
+ *       muloco_sync_status reports MULOCO_ETIMEOUT.  One-shot.
+ * After MULOCO_ETIMEOUT the context stays usable.  The step that timed out is incomplete: for
+ * the hidden matrices of the affected shape group the momentum has been advanced, but the
+ * parameters theta_k of some of its (worker, matrix) pairs have been updated, or partly
+ * updated, and others not, and nothing records which.  A caller that wants to continue
+ * restores theta_k and the momenta of that step from its own copy (a checkpoint of the
+ * caller-owned tensors plus muloco_get_state / muloco_set_state) and repeats the step. */
+enum { MULOCO_DEBUG_WAIT_LIMIT_NS = 1, MULOCO_DEBUG_WITHHOLD_COPY = 2 };
+MULOCO_API muloco_status muloco_debug_set(muloco_ctx* ctx, int32_t what, int64_t value);
+
 /* Waits for the stream and returns the device status word as a muloco_status
  * (MULOCO_OK, MULOCO_ENONFINITE, MULOCO_ETIMEOUT, MULOCO_ECUDA); clears it. */
 MULOCO_API muloco_status muloco_sync_status(muloco_ctx* ctx);

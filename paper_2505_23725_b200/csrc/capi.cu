@@ -31,7 +31,9 @@ struct TensorInfo {
 };
 
 struct WsLayout {   // byte offsets inside the workspace for one shape group
-  size_t x0, x1, a, b, partials, scales, total;
+  // fp32 engine: x0, x1, a, b are chunk-sized.  bf16 engine: x0 is the chunk-sized staged input and
+  // `ring` holds the intermediates of 2 * group matrices; `counters` counts finished tiles.
+  size_t x0, x1, a, b, ring, partials, scales, counters, total;
 };
 
 struct Group {
@@ -41,6 +43,7 @@ struct Group {
   int n_part = 0;
   int elt = 2;
   int mode = MULOCO_NS_BF16;   // engine that serves this group (see engine_for)
+  int ring_group = 1;          // bf16 engine: matrices per group of the work list (ring = 2 * ring_group slots)
   WsLayout ws;
   TcGroupPlan* plan = nullptr;
 };
@@ -76,19 +79,53 @@ int engine_for(int requested_mode, int64_t s) {
   return (requested_mode == MULOCO_NS_BF16 && s >= BF16_MIN_S) ? MULOCO_NS_BF16 : MULOCO_NS_FP32;
 }
 
-WsLayout make_layout(int64_t s, int64_t ldx, int64_t lds, int chunk, int n_part, int elt) {
+WsLayout make_layout(int64_t s, int64_t ldx, int64_t lds, int chunk, int n_part, int elt, int ring_group,
+                     int ns_steps) {
   WsLayout w;
+  memset(&w, 0, sizeof w);
   size_t off = 0;
   const size_t xb = align_up((size_t)chunk * s * ldx * elt, 1024);
-  const size_t sb = align_up((size_t)chunk * s * lds * elt, 1024);
   w.x0 = off; off += xb;
-  w.x1 = off; off += xb;
-  w.a = off; off += sb;
-  w.b = off; off += sb;
+  if (elt == 2) {
+    w.ring = off; off += tc_ring_bytes(s, ldx, lds, 2 * ring_group);
+  } else {
+    const size_t sb = align_up((size_t)chunk * s * lds * elt, 1024);
+    w.x1 = off; off += xb;
+    w.a = off; off += sb;
+    w.b = off; off += sb;
+  }
   w.partials = off; off += align_up((size_t)chunk * n_part * sizeof(float), 1024);
   w.scales = off; off += align_up((size_t)chunk * sizeof(float2), 1024);
+  w.counters = off; off += align_up((size_t)chunk * 3 * ns_steps * sizeof(int), 1024);
   w.total = off;
   return w;
+}
+
+// Matrices per workspace chunk: as many as the budget holds, then evened out so that
+// all chunks of a group have (nearly) the same size.
+int pick_chunk(int64_t count, size_t per_slot, size_t budget) {
+  int64_t ch = (int64_t)(budget / (per_slot ? per_slot : 1));
+  if (ch < 1) ch = 1;
+  if (ch >= count) return (int)std::max<int64_t>(count, 1);
+  const int64_t n_chunks = (count + ch - 1) / ch;
+  return (int)((count + n_chunks - 1) / n_chunks);
+}
+
+// Chunk size and ring size of a group of `count` same-shape matrices within `budget` bytes.
+void size_group(int64_t s, int64_t l, int64_t ldx, int64_t lds, int64_t count, size_t budget, int mode,
+                int ns_steps, int* chunk, int* ring_group) {
+  const int np = prologue_partials_per_matrix(s, l);
+  const int elt = (mode == MULOCO_NS_BF16) ? 2 : 4;
+  int rg = 1;
+  size_t fixed = 0;
+  if (elt == 2) {
+    rg = tc_group_size(s, (int)std::min<int64_t>(count, 1 << 30));
+    fixed = tc_ring_bytes(s, ldx, lds, 2 * rg);
+  }
+  const size_t per_slot = make_layout(s, ldx, lds, 1, np, elt, 0, ns_steps).total;
+  const size_t avail = budget > fixed + per_slot ? budget - fixed : per_slot;
+  *chunk = pick_chunk(count, per_slot, avail);
+  *ring_group = std::min(rg, *chunk);
 }
 
 }  // namespace
@@ -101,6 +138,8 @@ struct muloco_ctx {
   int n_sms = 148;
   std::string err;
   int* d_status = nullptr;
+  unsigned long long wait_limit_ns = 0;   // limit of the device-side waits of the bf16 engine (0: its default)
+  int debug_withhold = 0;                 // test hook, see muloco_debug_set
 
   std::vector<int> muon_ids, adam_ids;
   std::vector<Group> groups;
@@ -245,11 +284,11 @@ muloco_status setup_group(muloco_ctx* c, Group& g, char* ws, int mode) {
   g.mode = mode;
   g.elt = (mode == MULOCO_NS_BF16) ? 2 : 4;
   g.n_part = prologue_partials_per_matrix(g.s, g.l);
-  g.ws = make_layout(g.s, g.ldx, g.lds, g.chunk, g.n_part, g.elt);
+  g.ws = make_layout(g.s, g.ldx, g.lds, g.chunk, g.n_part, g.elt, g.ring_group, c->cfg.ns_steps);
   if (mode == MULOCO_NS_BF16) {
     char err[256] = {0};
-    g.plan = tc_plan_create(g.s, g.l, g.chunk, ws + g.ws.x0, ws + g.ws.x1, g.ldx, ws + g.ws.a,
-                            ws + g.ws.b, g.lds, err, sizeof err);
+    g.plan = tc_plan_create(g.s, g.l, g.chunk, ws + g.ws.x0, g.ldx, ws + g.ws.ring, g.lds, g.ring_group,
+                            reinterpret_cast<int*>(ws + g.ws.counters), c->cfg.ns_steps, err, sizeof err);
     if (!g.plan) return fail(c, MULOCO_ECUDA, "%s", err);
   }
   return MULOCO_OK;
@@ -273,42 +312,35 @@ muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_m
   NsIterArgs a;
   a.a = f.ns_a; a.b = f.ns_b; a.c = f.ns_c;
   a.mats = d_mats; a.sink_mode = sink_mode; a.status = c->d_status;
+  if (mode == MULOCO_NS_BF16) {
+    // one launch: every product of every iteration, the parameter update fused into the last one
+    a.scales = scales;
+    a.wait_limit_ns = c->wait_limit_ns;
+    a.debug_withhold = c->debug_withhold;
+    c->debug_withhold = 0;                       // one-shot
+    CK(tc_launch(c->st, g.plan, n_mats, a));
+    c->launches += 1;
+    CK(cudaGetLastError());
+    return MULOCO_OK;
+  }
   for (int it = 0; it < f.ns_steps; ++it) {
     const int xin = it & 1;
     const bool last = (it == f.ns_steps - 1);
+    float* Xin = reinterpret_cast<float*>(X[xin]);
+    float* Xout = reinterpret_cast<float*>(X[1 - xin]);
+    float* A = reinterpret_cast<float*>(ws + g.ws.a);
+    float* B = reinterpret_cast<float*>(ws + g.ws.b);
     a.scales = (it == 0) ? scales : nullptr;
-    if (mode == MULOCO_NS_BF16) {
-      CK(tc_launch(c->st, g.plan, GEMM_GRAM, n_mats, xin, a));
-      a.scales = nullptr;
-      CK(tc_launch(c->st, g.plan, GEMM_POLY, n_mats, xin, a));
-      a.scales = (it == 0) ? scales : nullptr;
-      CK(tc_launch(c->st, g.plan, last ? GEMM_FINAL : GEMM_APPLY, n_mats, xin, a));
-    } else {
-      float* Xin = reinterpret_cast<float*>(X[xin]);
-      float* Xout = reinterpret_cast<float*>(X[1 - xin]);
-      float* A = reinterpret_cast<float*>(ws + g.ws.a);
-      float* B = reinterpret_cast<float*>(ws + g.ws.b);
-      launch_ns_fp32(c->st, GEMM_GRAM, n_mats, g.s, g.l, Xin, g.ldx, A, B, g.lds, A, B, Xout, a);
-      a.scales = nullptr;
-      launch_ns_fp32(c->st, GEMM_POLY, n_mats, g.s, g.l, Xin, g.ldx, A, B, g.lds, A, B, Xout, a);
-      a.scales = (it == 0) ? scales : nullptr;
-      launch_ns_fp32(c->st, last ? GEMM_FINAL : GEMM_APPLY, n_mats, g.s, g.l, Xin, g.ldx, A, B, g.lds,
-                     A, B, Xout, a);
-    }
+    launch_ns_fp32(c->st, GEMM_GRAM, n_mats, g.s, g.l, Xin, g.ldx, A, B, g.lds, A, B, Xout, a);
+    a.scales = nullptr;
+    launch_ns_fp32(c->st, GEMM_POLY, n_mats, g.s, g.l, Xin, g.ldx, A, B, g.lds, A, B, Xout, a);
+    a.scales = (it == 0) ? scales : nullptr;
+    launch_ns_fp32(c->st, last ? GEMM_FINAL : GEMM_APPLY, n_mats, g.s, g.l, Xin, g.ldx, A, B, g.lds,
+                   A, B, Xout, a);
     c->launches += 3;
   }
   CK(cudaGetLastError());
   return MULOCO_OK;
-}
-
-// Matrices per workspace chunk: as many as the budget holds, then evened out so that
-// all chunks of a group have (nearly) the same size.
-int pick_chunk(int64_t count, size_t per_slot, size_t budget) {
-  int64_t ch = (int64_t)(budget / (per_slot ? per_slot : 1));
-  if (ch < 1) ch = 1;
-  if (ch >= count) return (int)std::max<int64_t>(count, 1);
-  const int64_t n_chunks = (count + ch - 1) / ch;
-  return (int)((count + n_chunks - 1) / n_chunks);
 }
 
 muloco_status build_sync_tables(muloco_ctx* c) {
@@ -508,10 +540,11 @@ MULOCO_API muloco_status muloco_create(const muloco_config* cfg, const muloco_te
   size_t need = 0;
   for (Group& g : c->groups) {
     const int np = prologue_partials_per_matrix(g.s, g.l);
-    const int elt = (engine_for(cfg->ns_mode, g.s) == MULOCO_NS_BF16) ? 2 : 4;
-    const size_t per_slot = make_layout(g.s, g.ldx, g.lds, 1, np, elt).total;
-    g.chunk = pick_chunk((int64_t)g.tensors.size() * K, per_slot, budget);
-    need = std::max(need, make_layout(g.s, g.ldx, g.lds, g.chunk, np, elt).total);
+    const int gmode = engine_for(cfg->ns_mode, g.s);
+    size_group(g.s, g.l, g.ldx, g.lds, (int64_t)g.tensors.size() * K, budget, gmode, cfg->ns_steps, &g.chunk,
+               &g.ring_group);
+    need = std::max(need, make_layout(g.s, g.ldx, g.lds, g.chunk, np, gmode == MULOCO_NS_BF16 ? 2 : 4,
+                                      g.ring_group, cfg->ns_steps).total);
   }
   if (need) {
     cudaError_t e = cudaMalloc(&c->ws, need);
@@ -862,15 +895,15 @@ MULOCO_API muloco_status muloco_newton_schulz(muloco_ctx* c, const void* X, int3
   const int elt = (ns_mode == MULOCO_NS_BF16) ? 2 : 4;
   const int64_t ldx = (l + 7) / 8 * 8, lds = (s + 7) / 8 * 8;
   const int np = prologue_partials_per_matrix(s, l);
-  const size_t per_slot = make_layout(s, ldx, lds, 1, np, elt).total;
   const size_t budget = c->cfg.workspace_bytes ? (size_t)c->cfg.workspace_bytes : ((size_t)6 << 30);
-  const int chunk = pick_chunk(batch, per_slot, budget);
+  int chunk = 1, ring_group = 1;
+  size_group(s, l, ldx, lds, batch, budget, ns_mode, c->cfg.ns_steps, &chunk, &ring_group);
   if (g.s != s || g.l != l || c->sa_mode != ns_mode || g.chunk != chunk || !c->sa_ws) {
     CK(cudaStreamSynchronize(c->st));
     destroy_group(g);
     g = Group();
-    g.s = s; g.l = l; g.ldx = ldx; g.lds = lds; g.chunk = chunk;
-    const size_t need = make_layout(s, ldx, lds, chunk, np, elt).total;
+    g.s = s; g.l = l; g.ldx = ldx; g.lds = lds; g.chunk = chunk; g.ring_group = ring_group;
+    const size_t need = make_layout(s, ldx, lds, chunk, np, elt, ring_group, c->cfg.ns_steps).total;
     if (need > c->sa_ws_bytes) {
       if (c->sa_ws) cudaFree(c->sa_ws);
       c->sa_ws = nullptr; c->sa_ws_bytes = 0;
@@ -1026,6 +1059,20 @@ MULOCO_API muloco_status muloco_get_timings(muloco_ctx* c, float* ms, int64_t* l
   if (launches) *launches = c->launches;
   c->launches = 0;
   return MULOCO_OK;
+}
+
+MULOCO_API muloco_status muloco_debug_set(muloco_ctx* c, int32_t what, int64_t value) {
+  if (!c) return MULOCO_EINVAL;
+  if (what == MULOCO_DEBUG_WAIT_LIMIT_NS) {
+    if (value < 0) return fail(c, MULOCO_EINVAL, "wait limit must be >= 0");
+    c->wait_limit_ns = (unsigned long long)value;
+    return MULOCO_OK;
+  }
+  if (what == MULOCO_DEBUG_WITHHOLD_COPY) {
+    c->debug_withhold = value != 0;
+    return MULOCO_OK;
+  }
+  return fail(c, MULOCO_EINVAL, "unknown debug switch %d", what);
 }
 
 MULOCO_API muloco_status muloco_sync_status(muloco_ctx* c) {

@@ -50,19 +50,27 @@ struct NsIterArgs {
   const MatDesc* mats;      // for GEMM_FINAL (sink)
   int sink_mode;
   int* status;
+  unsigned long long wait_limit_ns = 0;   // tensor-core engine: limit of every device-side wait (0: 2 s)
+  int debug_withhold = 0;                 // tensor-core engine, test hook: one operand copy is never issued
 };
 void launch_ns_fp32(cudaStream_t st, int kind, int n_mats, int64_t s, int64_t l, const float* X,
                     int64_t ldx, const float* A, const float* B, int64_t lds, float* Aout,
                     float* Bout, float* Xout, const NsIterArgs& args);
 
-// bf16 tensor-core engine (tcgen05 / TMEM / TMA); see ns_tc.cu.
-struct TcGroupPlan;   // opaque per-shape-group plan (tensor maps, tile lists)
-TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1, int64_t ldx,
-                            void* A, void* B, int64_t lds, char* err, size_t errlen);
+// bf16 tensor-core engine (tcgen05 / TMEM / TMA); see ns_tc.cu.  One launch runs all products of
+// all iterations for the matrices of a chunk; the staged input X0 is chunk-sized, the
+// intermediates live in a ring of 2 * group slots.
+struct TcGroupPlan;   // opaque per-shape-group plan (tensor maps, tile lists, work lists)
+// matrices per group of the work list for min-dimension s (never more than `chunk`)
+int tc_group_size(int64_t s, int chunk);
+// bytes of the ring (X', X'', A, B for n_slots matrices, bf16)
+size_t tc_ring_bytes(int64_t s, int64_t ldx, int64_t lds, int n_slots);
+// counters: chunk * 3 * ns_steps ints (zeroed by every launch)
+TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, int64_t ldx, void* ring, int64_t lds,
+                            int group, int* counters, int ns_steps, char* err, size_t errlen);
 void tc_plan_destroy(TcGroupPlan*);
-// runs one product for the first n_mats slots; xin selects which X buffer is the input (0/1)
-cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* plan, int kind, int n_mats, int xin,
-                      const NsIterArgs& args);
+// the whole iteration for the first n_mats matrices of the chunk (args.scales: per-matrix {r^2, r})
+cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* plan, int n_mats, const NsIterArgs& args);
 int tc_num_sms();
 // Encodes (into 128 bytes at `out_host`) the TMA descriptor of a rows x cols fp32 tensor for 32 x 32
 // boxes; swizzled for tensors stored s x l, plain for tensors stored l x s.  False when the tensor

@@ -2,14 +2,29 @@
 // accumulators in tensor memory, operands staged in shared memory by TMA
 // (128-byte swizzle), mbarrier pipeline, warp-specialised persistent CTAs.
 //
-// One launch computes one of the three products of a Newton-Schulz iteration
-// (Section 2, "Muon": X_j = p(X X^T) X, p(x) = a x + b x^3 + c x^5) for every
-// matrix of a chunk; tiles of all matrices form one linear work list:
+// ONE launch runs the whole iteration (Section 2, "Muon": X_j = p(X X^T) X,
+// p(x) = a x + b x^3 + c x^5, five times) for every matrix of a chunk.  Each
+// iteration is three products,
 //   GRAM  : A  = r^2 X X^T      symmetric: only the tiles on or above the diagonal are computed
 //   POLY  : B' = a I + b A + c A A   AND stored; a consumer fetches a block below the diagonal as
 //                               the transpose of its mirror image (an MN-major operand)
 //   APPLY : X' = r B' X  (= r (a X + b A X + c A A X); with a on B's diagonal the product needs no addend)
-//   FINAL : as APPLY, result goes to the parameter update / output sink
+//   FINAL : as APPLY in the last iteration, the result goes to the parameter update / output sink
+// and the tiles of all products of all matrices form one linear list of work items that the host
+// lays out (a table of blocks, one block = one product of a few matrices).  The list is ordered so
+// that a matrix's intermediates are consumed while they are still in L2: the matrices are taken
+// in groups of D, a group runs its 15 products one after the other over all its matrices, and the
+// intermediates (X', A, B') live in a small ring of 2 D slots that the next group but one reuses;
+// only the first Gram and the first apply read the staged input from its chunk-sized buffer.
+//
+// Work items go to the tile workers round-robin (item i to worker i mod W), every worker takes its
+// items in increasing order, and all workers are resident at once.  An item only depends on items
+// before it in the list: a product of matrix m needs all tiles of m's previous product (and the
+// first product of m needs the ring slot's previous user to be finished).  Finished tiles are
+// counted per (matrix, product) in global memory: every epilogue warp adds one (release) once its
+// part of the tile is in memory; the TMA producer (and, for the polynomial's addend, the epilogue)
+// waits (acquire) until the count of the product it reads is complete.  The item with the smallest
+// index that is not finished always has its inputs ready, so the list drains.
 // Operand forms: GRAM/POLY multiply a row-major matrix by its own transpose
 // (both operands K-major); APPLY needs X with the contraction index as the slow
 // axis, i.e. an MN-major B operand, so no transposed copy of X is ever made.
@@ -28,15 +43,16 @@
 // the accumulator each).  Two accumulators alternate so the epilogue of one
 // tile overlaps the main loop of the next.  The epilogue goes through shared
 // memory: the addend (A for POLY) arrives by TMA, results leave as
-// bulk tensor stores of whole 32 x 64 blocks (and, for the symmetric products,
-// of the transposed block), so global memory only sees full lines.
-// Every wait is bounded: when one runs out the kernel raises ST_TIMEOUT, all
-// roles leave their loops, and the CTA frees its tensor memory and returns.
+// bulk tensor stores of whole 32 x 64 blocks, so global memory only sees full lines.
+// Every wait is bounded (on a barrier or on a counter): when one runs out the kernel raises
+// ST_TIMEOUT, all roles leave their loops, the CTA frees its tensor memory and returns; the other
+// CTAs see the flag in the status word at their next counter wait and leave as well.
 #include <cuda.h>
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
+#include <map>
 #include <vector>
 
 #include "internal.h"
@@ -50,34 +66,68 @@ constexpr int BM = 128;          // rows per CTA (one CTA's share of UMMA M)
 constexpr int BK = 64;           // k slab per stage (64 bf16 = one 128-byte swizzle row)
 constexpr int UMMA_K = 16;
 constexpr int TC_THREADS = 192;
-// Pipeline depth is a template parameter; every product runs 5 stages beside four staging blocks
-// per epilogue warp (GRAM, APPLY: results; POLY: addend + results; FINAL: the parameter ring).
+constexpr int TC_STAGES = 5;
+// Five pipeline stages beside four staging blocks per epilogue warp (GRAM, APPLY: results; POLY:
+// addend + results; FINAL: the parameter ring).
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;        // 16 KB: 128 rows x 64 k
 constexpr uint32_t B_STAGE_BYTES = 128 * BK * 2;       // 16 KB: this CTA's 128 columns of the right operand
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr uint32_t EPI_BLOCK_BYTES = 32 * 64 * 2;      // one 32 x 64 bf16 block
-__host__ __device__ constexpr uint32_t epi_warp_bytes(int) { return 4u * EPI_BLOCK_BYTES; }
-__host__ __device__ constexpr uint32_t smem_bytes(int nstg) {
-  return (uint32_t)nstg * STAGE_BYTES + 4u * epi_warp_bytes(nstg) + 1024u;   // + alignment slack
-}
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+constexpr uint32_t EPI_WARP_BYTES = 4u * EPI_BLOCK_BYTES;
+constexpr uint32_t TC_SMEM_BYTES = (uint32_t)TC_STAGES * STAGE_BYTES + 4u * EPI_WARP_BYTES + 1024u;   // + alignment slack
+
+// One block of the work list: the tiles of one product (`ph` = 3 * iteration + {0 Gram, 1 polynomial,
+// 2 apply}) of the matrices [mat0, mat0 + n_mats) of the chunk, matrix-major.
+struct TcBlock {
+  int first_item, n_items;
+  int kind, ph;
+  int mat0, n_mats;
+  int pad0, pad1;
+};
+
+// Tensor maps of one shape group.  X0 is the chunk-sized staged input (third coordinate: matrix of
+// the chunk); XA, XB, A, B are the ring (third coordinate: slot).  _K: K-major operand boxes
+// (64 x 128); _MN: MN-major operand boxes (one 4-D copy per slab when the column count allows it,
+// else 64 x 64 boxes); _IO: 64 x 32 boxes for addend loads and result stores.
+enum MapId : int {
+  MAP_X0_K = 0, MAP_XA_K, MAP_XB_K,
+  MAP_X0_MN, MAP_XA_MN, MAP_XB_MN,
+  MAP_XA_IO, MAP_XB_IO,
+  MAP_A_K, MAP_A_MN, MAP_A_IO,
+  MAP_B_K, MAP_B_MN, MAP_B_IO,
+  N_MAPS
+};
+struct TcMaps {
+  CUtensorMap m[N_MAPS];
+};
 
 struct TcParams {
-  int kind;
-  int n_mats;
-  int M, N, Kd;
-  int n_tiles_per_mat;
-  const int2* tiles;          // (tile row, tile col) in units of 128*CG
+  const TcBlock* blocks;
+  int n_blocks, total_items;
+  const int2* tiles_sym;      // (tile row, tile col) in units of 128*CG, tiles on or above the diagonal
+  const int2* tiles_full;     // all tiles of the s x l result
+  int n_sym, n_full;
+  int s, l;
+  int last_ph;                // 3 * ns_steps - 1: the product whose result goes to the sink
   float a, b, c;
-  const float2* scales;
-  const MatDesc* mats;
+  const float2* scales;       // per matrix of the chunk {r^2, r}; applied in the first iteration
+  const MatDesc* mats;        // per matrix of the chunk (sink)
   int sink_mode;
-  int a_tri, b_tri;           // left / right operand is a symmetric matrix of which only the tiles on
-                              // or above the diagonal are stored
-  int b_wide, s_wide;         // tmB (MN-major right operand) / tmS (mirror-image boxes) is the 4-D form:
-                              // one copy brings both 64-column atoms (128 operand rows x 64 k) of a slab
-  int64_t s, l;
+  int x_wide, s_wide;         // the _MN maps of X / of A and B are the 4-D form (both 64-column atoms of a slab in one copy)
+  int n_slots;
+  int* counters;              // [chunk][cw]: epilogue warps that have finished product ph of matrix m
+  int cw;
   int* status;
+  unsigned long long wait_limit_ns;
+  int debug_withhold;         // test hook: worker 0 never issues the first operand copy of its first item
+};
+
+// One work item, as every role decodes it.
+struct Item {
+  int kind, ph, it;           // product, its index 3 * it + {0, 1, 2}, iteration
+  int m, slot;                // matrix of the chunk, ring slot
+  int2 tt;                    // tile
+  int N, Kd;                  // result columns, contraction length
 };
 
 // ----------------------------- PTX wrappers --------------------------------
@@ -128,7 +178,8 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait ran out, or another did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (;;) {
@@ -136,7 +187,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+    if (global_timer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       return false;
     }
@@ -286,18 +337,81 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
   asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
+// ----------------------------- work-list helpers ----------------------------
+__device__ __forceinline__ Item decode_item(const TcParams& p, int item, int& cur) {
+  // items of one worker increase, so the block cursor only moves forward
+  const int4* bt = reinterpret_cast<const int4*>(p.blocks);
+  int4 b0 = __ldg(bt + 2 * cur);
+  while (item >= b0.x + b0.y) {
+    ++cur;
+    b0 = __ldg(bt + 2 * cur);
+  }
+  const int mat0 = __ldg(reinterpret_cast<const int*>(p.blocks) + 8 * cur + 4);
+  Item q;
+  q.kind = b0.z;
+  q.ph = b0.w;
+  q.it = q.ph / 3;
+  const bool sym = q.kind <= GEMM_POLY;
+  const int tpm = sym ? p.n_sym : p.n_full;
+  const int r = item - b0.x;
+  const int ml = r / tpm;
+  q.m = mat0 + ml;
+  q.slot = q.m % p.n_slots;
+  q.tt = (sym ? p.tiles_sym : p.tiles_full)[r - ml * tpm];
+  q.N = sym ? p.s : p.l;
+  q.Kd = (q.kind == GEMM_GRAM) ? p.l : p.s;
+  return q;
+}
+
+__device__ __forceinline__ int ld_acquire(const int* ptr) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+// Waits until the product this item reads is complete (all tiles of the matrix's previous product;
+// for a matrix's first product: the last product of the ring slot's previous user).  Called by one
+// thread.  Returns false when the CTA is aborting or another CTA has raised ST_TIMEOUT.
+template <int CG>
+__device__ __forceinline__ bool dep_wait(const TcParams& p, const Item& q, volatile int* abort_flag) {
+  const int* cnt;
+  int need;
+  if (q.ph > 0) {
+    cnt = p.counters + (int64_t)q.m * p.cw + (q.ph - 1);
+    need = (((q.ph - 1) % 3 == 2) ? p.n_full : p.n_sym) * 4 * CG;
+  } else if (q.m >= p.n_slots) {
+    cnt = p.counters + (int64_t)(q.m - p.n_slots) * p.cw + p.last_ph;
+    need = p.n_full * 4 * CG;
+  } else {
+    return true;
+  }
+  if (ld_acquire(cnt) < need) {
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+      if (ld_acquire(cnt) >= need) break;
+      if (*abort_flag) return false;
+      if (ld_acquire(p.status) & ST_TIMEOUT) { *abort_flag = 1; return false; }
+      if (global_timer_ns() - t0 > p.wait_limit_ns) { *abort_flag = 1; return false; }
+      __nanosleep(64);
+    }
+  }
+  // what the other CTAs wrote through the async proxy is read through the async proxy next
+  asm volatile("fence.proxy.async;" ::: "memory");
+  return true;
+}
+
+// One epilogue warp has finished its part of a tile (its stores are complete): count it.
+__device__ __forceinline__ void signal_done(const TcParams& p, const Item& q) {
+  int* cnt = p.counters + (int64_t)q.m * p.cw + q.ph;
+  asm volatile("fence.proxy.async;" ::: "memory");
+  asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
+}
+
 // ------------------------------- the kernel --------------------------------
-// tmA/tmB : operand loads (left: K-major 64 x 128 boxes; right: K-major 64 x 128 or, for B_MN,
-//           MN-major 64 x 64 boxes)
-// tmC     : addend loads, 64 x 32 boxes (POLY: A; unused by the other products)
-// tmD     : result stores, 64 x 32 boxes, 128-byte swizzle
-// tmS     : 64 x 64 boxes over the symmetric operand (POLY: A, APPLY/FINAL: B) for the k slabs
-//           whose block lies below the diagonal and is read from its mirror image
-template <int CG, bool B_MN, int STAGES>
+template <int CG>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-             const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
-             const __grid_constant__ CUtensorMap tmS, const TcParams p) {
+ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+  constexpr int STAGES = TC_STAGES;
   constexpr int BN = 128 * CG;                 // accumulator columns = tile columns
   constexpr int TM = 128 * CG;                 // tile rows (over the CTA pair)
   constexpr uint32_t TMEM_COLS = 2 * BN;
@@ -318,17 +432,12 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   const int unit = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // tile worker index
   const int n_units = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const int total_tiles = p.n_mats * p.n_tiles_per_mat;
-  const int num_kb = (p.Kd + BK - 1) / BK;
-  const bool sym = (p.kind == GEMM_GRAM || p.kind == GEMM_POLY);
+  const uint64_t limit = p.wait_limit_ns;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmS) : "memory");
+#pragma unroll 1
+    for (int i = 0; i < N_MAPS; ++i) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[i]) : "memory");
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
@@ -360,45 +469,77 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const uint32_t full0_bar = (CG == 2) ? map_to_rank(full0, 0) : full0;
       uint32_t stage = 0, phase = 0;
       bool alive = true;
-      for (int tile = unit; tile < total_tiles && alive; tile += n_units) {
-        const int mat = tile / p.n_tiles_per_mat;
-        const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
-        const bool same = sym && (tt.x == tt.y);     // diagonal tile: right slab == left slab
-        const int a_row = BM * (CG * tt.x + (int)rank);
-        const int b_off = TM * tt.y + 128 * (int)rank;
+      int cur = 0;
+      bool withhold = (p.debug_withhold != 0) && (unit == 0);
+      for (int item = unit; item < p.total_items && alive; item += n_units) {
+        const Item q = decode_item(p, item, cur);
+        if (!dep_wait<CG>(p, q, &abort_flag)) break;
+        const bool sym = q.kind <= GEMM_POLY;
+        const bool b_is_x = q.kind >= GEMM_APPLY;             // right operand: X, MN-major
+        const bool same = sym && (q.tt.x == q.tt.y);          // diagonal tile: right slab == left slab
+        const int xsel = (q.it == 0) ? 0 : ((q.it & 1) ? 1 : 2);
+        const CUtensorMap* mA;
+        const CUtensorMap* mB;
+        const CUtensorMap* mS;
+        int zA, zB;
+        if (q.kind == GEMM_GRAM) {
+          mA = mB = &maps.m[MAP_X0_K + xsel];
+          zA = zB = (q.it == 0) ? q.m : q.slot;
+          mS = mA;
+        } else if (q.kind == GEMM_POLY) {
+          mA = mB = &maps.m[MAP_A_K];
+          zA = zB = q.slot;
+          mS = &maps.m[MAP_A_MN];
+        } else {
+          mA = &maps.m[MAP_B_K];
+          zA = q.slot;
+          mB = &maps.m[MAP_X0_MN + xsel];
+          zB = (q.it == 0) ? q.m : q.slot;
+          mS = &maps.m[MAP_B_MN];
+        }
+        const int a_row = BM * (CG * q.tt.x + (int)rank);
+        const int b_off = TM * q.tt.y + 128 * (int)rank;
         const uint32_t cta_bytes = A_STAGE_BYTES + (same ? 0u : B_STAGE_BYTES);
         // blocks of a symmetric operand below the diagonal are not stored: their k slab is fetched
-        // from the mirror image as two 64 x 64 boxes (k rows, 64 operand rows each)
-        const int ka_mn = p.a_tri ? (TM / BK) * tt.x : 0;
-        const int kb_mn = p.b_tri ? (TM / BK) * tt.y : 0;
+        // from the mirror image as two 64-column atoms (k rows, 64 operand rows each)
+        const int ka_mn = (q.kind != GEMM_GRAM) ? (TM / BK) * q.tt.x : 0;
+        const int kb_mn = (q.kind == GEMM_POLY) ? (TM / BK) * q.tt.y : 0;
+        const int num_kb = (q.Kd + BK - 1) / BK;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(empty0 + stage * 8u, phase ^ 1u, &abort_flag)) { alive = false; break; }
+          if (!mbar_wait(empty0 + stage * 8u, phase ^ 1u, &abort_flag, limit)) { alive = false; break; }
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_STAGE_BYTES;
           const uint32_t bar = full0_bar + stage * 8u;
+          if (withhold) {
+            // test hook: nothing is expected and nothing is copied for this stage, so the MMA
+            // issuer's wait for it runs out
+            withhold = false;
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           if (CG == 1) mbar_expect_tx(bar, cta_bytes);
           else if (rank == 0) mbar_expect_tx(full0 + stage * 8u, 2u * cta_bytes);
-          auto load = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1) {
-            if (CG == 1) tma_load_3d(dst, map, bar, c0, c1, mat);
-            else tma_load_3d_pair(dst, map, bar, c0, c1, mat);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1, int z) {
+            if (CG == 1) tma_load_3d(dst, map, bar, c0, c1, z);
+            else tma_load_3d_pair(dst, map, bar, c0, c1, z);
           };
           // an MN-major slab = two 64-column atoms of 64 k rows: one 4-D copy, or two 64 x 64 boxes
-          auto load_mn = [&](uint32_t dst, const CUtensorMap* map, bool wide, int col0, int k) {
+          auto load_mn = [&](uint32_t dst, const CUtensorMap* map, bool wide, int col0, int k, int z) {
             if (wide) {
-              if (CG == 1) tma_load_4d(dst, map, bar, 0, k, col0 >> 6, mat);
-              else tma_load_4d_pair(dst, map, bar, 0, k, col0 >> 6, mat);
+              if (CG == 1) tma_load_4d(dst, map, bar, 0, k, col0 >> 6, z);
+              else tma_load_4d_pair(dst, map, bar, 0, k, col0 >> 6, z);
             } else {
-              load(dst, map, col0, k);
-              load(dst + BK * 128, map, col0 + 64, k);
+              load(dst, map, col0, k, z);
+              load(dst + BK * 128, map, col0 + 64, k, z);
             }
           };
           const int k0 = kb * BK;
-          if (kb >= ka_mn) load(sa, &tmA, k0, a_row);
-          else load_mn(sa, &tmS, p.s_wide != 0, a_row, k0);
+          if (kb >= ka_mn) load(sa, mA, k0, a_row, zA);
+          else load_mn(sa, mS, p.s_wide != 0, a_row, k0, q.slot);
           if (!same) {
-            if (B_MN) load_mn(sb, &tmB, p.b_wide != 0, b_off, k0);
-            else if (kb >= kb_mn) load(sb, &tmB, k0, b_off);
-            else load_mn(sb, &tmS, p.s_wide != 0, b_off, k0);
+            if (b_is_x) load_mn(sb, mB, p.x_wide != 0, b_off, k0, zB);
+            else if (kb >= kb_mn) load(sb, mB, k0, b_off, zB);
+            else load_mn(sb, mS, p.s_wide != 0, b_off, k0, q.slot);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -426,20 +567,22 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       uint32_t stage = 0, phase = 0;
       int local_tile = 0;
       bool alive = true;
-      for (int tile = unit; tile < total_tiles && alive; tile += n_units, ++local_tile) {
-        const int mat = tile / p.n_tiles_per_mat;
-        const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
-        const bool same = sym && (tt.x == tt.y);
+      int cur = 0;
+      for (int item = unit; item < p.total_items && alive; item += n_units, ++local_tile) {
+        const Item q = decode_item(p, item, cur);
+        const bool sym = q.kind <= GEMM_POLY;
+        const bool same = sym && (q.tt.x == q.tt.y);
+        const int num_kb = (q.Kd + BK - 1) / BK;
         // k slabs below these indices come from the mirror image (MN-major), as staged by the producer
-        const int ka_mn = p.a_tri ? (TM / BK) * tt.x : 0;
-        const int kb_mn = B_MN ? num_kb : (p.b_tri ? (TM / BK) * tt.y : 0);
+        const int ka_mn = (q.kind != GEMM_GRAM) ? (TM / BK) * q.tt.x : 0;
+        const int kb_mn = (q.kind >= GEMM_APPLY) ? num_kb : ((q.kind == GEMM_POLY) ? (TM / BK) * q.tt.y : 0);
         const uint32_t acc = (uint32_t)local_tile & 1u;
         const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
         const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
-        if (!mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, &abort_flag)) break;
+        if (!mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, &abort_flag, limit)) break;
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(full0 + stage * 8u, phase, &abort_flag)) { alive = false; break; }
+          if (!mbar_wait(full0 + stage * 8u, phase, &abort_flag, limit)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = same ? sa : sa + A_STAGE_BYTES;
@@ -468,61 +611,82 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // -------------------------------- epilogue --------------------------------
     const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter+32)
     const int ew = warp - 2;               // staging slot of this warp
-    const uint32_t epi = smem_base + STAGES * STAGE_BYTES + (uint32_t)ew * epi_warp_bytes(STAGES);
+    const uint32_t epi = smem_base + STAGES * STAGE_BYTES + (uint32_t)ew * EPI_WARP_BYTES;
     // staging blocks of this warp: addend 0/1 (when there is one), then results 0/1
     auto cin_buf = [&](uint32_t b) { return epi + b * EPI_BLOCK_BYTES; };
-    const uint32_t o_first = (p.kind == GEMM_GRAM) ? 0u : 2u;     // the addend blocks come first when there are any
-    auto out_buf = [&](uint32_t b) { return epi + (o_first + b) * EPI_BLOCK_BYTES; };
     const uint32_t cin_bar0 = smem_u32(&bar_cin[ew][0]);
     auto cin_bar = [&](uint32_t b) { return cin_bar0 + b * 8u; };
-    // Only the polynomial has an addend (b A).  Its epilogue also adds a to the diagonal, B' = B + a I,
-    // so that the third product of the iteration, a X + B X = B' X, needs none.
-    const bool has_cin = (p.kind == GEMM_POLY);
-    const bool stores = (p.kind != GEMM_FINAL);
     // parameter update through TMA: a ring of four 32 x 32 fp32 blocks, the whole staging space of
     // the warp (the final product has no addend and stages no results)
     auto w_buf = [&](uint32_t b) { return epi + b * EPI_BLOCK_BYTES; };
     const uint32_t w_bar0 = smem_u32(&bar_w[ew][0]);
     auto w_bar = [&](uint32_t b) { return w_bar0 + b * 8u; };
-    const bool upd = (p.kind == GEMM_FINAL && p.sink_mode == SINK_UPDATE_W);
     uint32_t w_issued = 0, w_used = 0;
     uint32_t cin_issued = 0, cin_used = 0, st_count = 0, t_count = 0;
     int local_tile = 0;
     bool alive = true;
-    for (int tile = unit; tile < total_tiles && alive; tile += n_units, ++local_tile) {
+    int cur = 0;
+    int prev_kind = -1;
+    for (int item = unit; item < p.total_items && alive; item += n_units, ++local_tile) {
+      const Item q = decode_item(p, item, cur);
       const int acc = local_tile & 1;
       const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
-      const int mat = tile / p.n_tiles_per_mat;
-      const int2 tt = p.tiles[tile - mat * p.n_tiles_per_mat];
+      const int2 tt = q.tt;
+      const int mat = q.m;
+      // Only the polynomial has an addend (b A).  Its epilogue also adds a to the diagonal, B' = B + a I,
+      // so that the third product of the iteration, a X + B X = B' X, needs none.
+      const bool has_cin = (q.kind == GEMM_POLY);
+      const bool stores = (q.kind != GEMM_FINAL);
+      const bool upd = (q.kind == GEMM_FINAL && p.sink_mode == SINK_UPDATE_W);
+      const uint32_t o_first = (q.kind == GEMM_GRAM || q.kind == GEMM_APPLY) ? 0u : 2u;   // addend blocks come first
+      auto out_buf = [&](uint32_t b) { return epi + (o_first + b) * EPI_BLOCK_BYTES; };
+      const CUtensorMap* mC = &maps.m[MAP_A_IO];
+      const CUtensorMap* mD = (q.kind == GEMM_GRAM) ? &maps.m[MAP_A_IO]
+                              : (q.kind == GEMM_POLY) ? &maps.m[MAP_B_IO]
+                              : &maps.m[(q.it & 1) ? MAP_XB_IO : MAP_XA_IO];
+      if (q.kind != prev_kind) {
+        // the staging space is laid out per product: everything the previous product handed to the
+        // bulk stores has been read before it is reused under another layout
+        if (lane == 0) bulk_wait_read_0();
+        __syncwarp();
+        prev_kind = q.kind;
+      }
       const int rb = CG * tt.x + (int)rank;                 // 128-row block of this CTA
       const int gi0 = rb * BM + quarter * 32;               // first row of this warp
       const int gi = gi0 + lane;
-      const bool row_ok = gi < p.M;
+      const bool row_ok = gi < p.s;
       // 64-column blocks of this tile that this warp has to produce
       uint32_t todo = 0;
-      if (gi0 < p.M) {
+      if (gi0 < p.s) {
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int gj0 = TM * tt.y + c * 64;
-          if (gj0 < p.N) todo |= 1u << c;
+          if (gj0 < q.N) todo |= 1u << c;
         }
       }
       auto issue_cin = [&](int c) {
         if (lane == 0) {
           const uint32_t b = cin_issued & 1u;
           mbar_expect_tx(cin_bar(b), EPI_BLOCK_BYTES);
-          tma_load_3d(cin_buf(b), &tmC, cin_bar(b), TM * tt.y + c * 64, gi0, mat);
+          tma_load_3d(cin_buf(b), mC, cin_bar(b), TM * tt.y + c * 64, gi0, q.slot);
         }
         ++cin_issued;
       };
-      if (has_cin && todo) issue_cin(__ffs(todo) - 1);
+      if (has_cin && todo) {
+        // the addend is the Gram matrix of this iteration: wait until all of its tiles are in memory
+        int ok = 1;
+        if (lane == 0) ok = dep_wait<CG>(p, q, &abort_flag) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) { alive = false; break; }
+        issue_cin(__ffs(todo) - 1);
+      }
       // fused parameter update: the old parameters come in as 32 x 32 blocks, two steps ahead
       MatDesc dsc;
       dsc.wmap = nullptr; dsc.transposed = 0; dsc.lr_eff = 0.f; dsc.wd_term = 0.f;
       if (upd) dsc = p.mats[mat];
       const bool use_tma = upd && dsc.wmap != nullptr && todo != 0;
       int n_hb = 0;                                      // 32-column blocks of this warp in this tile
-      if (use_tma) n_hb = min(2 * NCH, (p.N - TM * tt.y + 31) >> 5);
+      if (use_tma) n_hb = min(2 * NCH, (q.N - TM * tt.y + 31) >> 5);
       auto issue_w = [&](int hb) {
         if (lane == 0) {
           const uint32_t b = w_issued & 3u;
@@ -542,12 +706,12 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (lane == 0) bulk_wait_read_0();               // plain path reuses the staging space
         __syncwarp();
       }
-      if (!mbar_wait(smem_u32(&bar_tfull[acc]), acc_phase, &abort_flag)) alive = false;
+      if (!mbar_wait(smem_u32(&bar_tfull[acc]), acc_phase, &abort_flag, limit)) alive = false;
       alive = __all_sync(0xffffffffu, alive);
       if (!alive) break;
       tc_fence_after();
       float sc = 1.f;
-      if (p.scales) sc = (p.kind == GEMM_GRAM) ? p.scales[mat].x : p.scales[mat].y;
+      if (p.scales && q.it == 0 && q.kind != GEMM_POLY) sc = (q.kind == GEMM_GRAM) ? p.scales[mat].x : p.scales[mat].y;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
       while (todo) {
@@ -556,7 +720,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int gj0 = TM * tt.y + c * 64;
         if (has_cin) {
           if (todo) issue_cin(__ffs(todo) - 1);
-          bool ok = mbar_wait(cin_bar(cin_used & 1u), (cin_used >> 1) & 1u, &abort_flag);
+          bool ok = mbar_wait(cin_bar(cin_used & 1u), (cin_used >> 1) & 1u, &abort_flag, limit);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) { alive = false; break; }
         }
@@ -576,12 +740,12 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           if (has_cin) {
             float add[32];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const uint4 u = lds128(cbuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q) ^ (lane & 7)) << 4));
-              add[q * 8 + 0] = bf16_lo(u.x); add[q * 8 + 1] = bf16_hi(u.x);
-              add[q * 8 + 2] = bf16_lo(u.y); add[q * 8 + 3] = bf16_hi(u.y);
-              add[q * 8 + 4] = bf16_lo(u.z); add[q * 8 + 5] = bf16_hi(u.z);
-              add[q * 8 + 6] = bf16_lo(u.w); add[q * 8 + 7] = bf16_hi(u.w);
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const uint4 u = lds128(cbuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q4) ^ (lane & 7)) << 4));
+              add[q4 * 8 + 0] = bf16_lo(u.x); add[q4 * 8 + 1] = bf16_hi(u.x);
+              add[q4 * 8 + 2] = bf16_lo(u.y); add[q4 * 8 + 3] = bf16_hi(u.y);
+              add[q4 * 8 + 4] = bf16_lo(u.z); add[q4 * 8 + 5] = bf16_hi(u.z);
+              add[q4 * 8 + 6] = bf16_lo(u.w); add[q4 * 8 + 7] = bf16_hi(u.w);
             }
             const int dcol = gi - (gj0 + h * 32);        // this lane's diagonal element, if it is in the block
 #pragma unroll
@@ -598,27 +762,27 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             // l x s it is the tile's row axis, which the lanes already hold.
             const int gjh = gj0 + h * 32;
             if (use_tma) {
-              if (gjh < p.N) {
+              if (gjh < q.N) {
                 const int hb = 2 * c + h;
                 if (lane == 0) bulk_wait_read_1();       // the block stored two steps ago has left the ring
                 __syncwarp();
                 if (hb + 2 < n_hb) issue_w(hb + 2);
-                bool ok = mbar_wait(w_bar(w_used & 3u), (w_used >> 2) & 1u, &abort_flag);
+                bool ok = mbar_wait(w_bar(w_used & 3u), (w_used >> 2) & 1u, &abort_flag, limit);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { alive = false; break; }
                 const uint32_t wb = w_buf(w_used & 3u);
                 if (!dsc.transposed) {
                   // block rows are tile rows: each lane owns one 128-byte row (swizzled)
 #pragma unroll
-                  for (int q = 0; q < 8; ++q) {
-                    const uint32_t ad = wb + (uint32_t)lane * 128u + ((uint32_t)(q ^ (lane & 7)) << 4);
+                  for (int q4 = 0; q4 < 8; ++q4) {
+                    const uint32_t ad = wb + (uint32_t)lane * 128u + ((uint32_t)(q4 ^ (lane & 7)) << 4);
                     uint4 u = lds128(ad);
                     float w0 = __uint_as_float(u.x), w1 = __uint_as_float(u.y), w2 = __uint_as_float(u.z),
                           w3 = __uint_as_float(u.w);
-                    w0 = fmaf(-dsc.lr_eff, f[q * 4 + 0], fmaf(-dsc.wd_term, w0, w0));
-                    w1 = fmaf(-dsc.lr_eff, f[q * 4 + 1], fmaf(-dsc.wd_term, w1, w1));
-                    w2 = fmaf(-dsc.lr_eff, f[q * 4 + 2], fmaf(-dsc.wd_term, w2, w2));
-                    w3 = fmaf(-dsc.lr_eff, f[q * 4 + 3], fmaf(-dsc.wd_term, w3, w3));
+                    w0 = fmaf(-dsc.lr_eff, f[q4 * 4 + 0], fmaf(-dsc.wd_term, w0, w0));
+                    w1 = fmaf(-dsc.lr_eff, f[q4 * 4 + 1], fmaf(-dsc.wd_term, w1, w1));
+                    w2 = fmaf(-dsc.lr_eff, f[q4 * 4 + 2], fmaf(-dsc.wd_term, w2, w2));
+                    w3 = fmaf(-dsc.lr_eff, f[q4 * 4 + 3], fmaf(-dsc.wd_term, w3, w3));
                     sts128(ad, make_uint4(__float_as_uint(w0), __float_as_uint(w1), __float_as_uint(w2),
                                           __float_as_uint(w3)));
                   }
@@ -640,20 +804,20 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 }
                 ++w_used;
               }
-            } else if (gjh < p.N) {
+            } else if (gjh < q.N) {
               const MatDesc d = p.mats[mat];
-              const bool full = (gi0 + 32 <= p.M) && (gjh + 32 <= p.N);
+              const bool full = (gi0 + 32 <= p.s) && (gjh + 32 <= q.N);
               if (full) {
                 float o[32];
                 int64_t base, stride;
                 if (!d.transposed) {
-                  const uint32_t tb = out_buf(t_count & 1u);
+                  const uint32_t tb = epi + (2u + (t_count & 1u)) * EPI_BLOCK_BYTES;
                   ++t_count;
 #pragma unroll
-                  for (int q = 0; q < 8; ++q)
-                    sts128(tb + (uint32_t)lane * 128u + ((uint32_t)(q ^ (lane & 7)) << 4),
-                           make_uint4(__float_as_uint(f[q * 4 + 0]), __float_as_uint(f[q * 4 + 1]),
-                                      __float_as_uint(f[q * 4 + 2]), __float_as_uint(f[q * 4 + 3])));
+                  for (int q4 = 0; q4 < 8; ++q4)
+                    sts128(tb + (uint32_t)lane * 128u + ((uint32_t)(q4 ^ (lane & 7)) << 4),
+                           make_uint4(__float_as_uint(f[q4 * 4 + 0]), __float_as_uint(f[q4 * 4 + 1]),
+                                      __float_as_uint(f[q4 * 4 + 2]), __float_as_uint(f[q4 * 4 + 3])));
                   __syncwarp();
 #pragma unroll
                   for (int r = 0; r < 32; ++r)
@@ -687,19 +851,19 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
               } else if (row_ok) {
 #pragma unroll
                 for (int e = 0; e < 32; ++e)
-                  if (gjh + e < p.N) sink_element(d, p.sink_mode, p.s, p.l, gi, gjh + e, f[e]);
+                  if (gjh + e < q.N) sink_element(d, p.sink_mode, p.s, p.l, gi, gjh + e, f[e]);
               }
             }
           } else {
-            // ---- stage the bf16 block (and its transpose) for the bulk stores ----
+            // ---- stage the bf16 block for the bulk store ----
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q4 = 0; q4 < 4; ++q4) {
               uint4 u;
-              u.x = pack_bf16x2(f[q * 8 + 0], f[q * 8 + 1]);
-              u.y = pack_bf16x2(f[q * 8 + 2], f[q * 8 + 3]);
-              u.z = pack_bf16x2(f[q * 8 + 4], f[q * 8 + 5]);
-              u.w = pack_bf16x2(f[q * 8 + 6], f[q * 8 + 7]);
-              sts128(obuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q) ^ (lane & 7)) << 4), u);
+              u.x = pack_bf16x2(f[q4 * 8 + 0], f[q4 * 8 + 1]);
+              u.y = pack_bf16x2(f[q4 * 8 + 2], f[q4 * 8 + 3]);
+              u.z = pack_bf16x2(f[q4 * 8 + 4], f[q4 * 8 + 5]);
+              u.w = pack_bf16x2(f[q4 * 8 + 6], f[q4 * 8 + 7]);
+              sts128(obuf + (uint32_t)lane * 128u + ((uint32_t)((h * 4 + q4) ^ (lane & 7)) << 4), u);
             }
           }
         }
@@ -709,7 +873,7 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_3d(&tmD, obuf, gj0, gi0, mat);
+            tma_store_3d(mD, obuf, gj0, gi0, q.slot);
             bulk_commit();
           }
           ++st_count;
@@ -723,6 +887,11 @@ ns_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       if (lane == 0) {
         const uint32_t te = smem_u32(&bar_tempty[acc]);
         mbar_arrive_cluster(CG == 2 ? map_to_rank(te, 0) : te);
+        // This warp's part of the tile: for a stored product its results are in memory once the
+        // bulk stores have completed; the final product only has to have read its operands, which
+        // it has (its accumulator was complete), so the ring slot may be reused.
+        if (stores) bulk_wait_all();
+        signal_done(p, q);
       }
     }
     bulk_wait_all();
@@ -813,18 +982,14 @@ bool tc_encode_w_map(void* out_host, void* base, int64_t rows, int64_t cols, int
 
 namespace {
 
-struct Maps5 {
-  const CUtensorMap *a, *b, *c, *d, *t;
-};
-
 // Number of tile workers (CTAs for CG = 1, CTA pairs for CG = 2) that can be resident at once.
-template <int CG, bool B_MN, int NSTG>
+template <int CG>
 int resident_units(int n_sms, cudaError_t* err) {
   static int cached = 0;
   *err = cudaSuccess;
   if (cached) return cached;
-  cudaError_t e = cudaFuncSetAttribute(ns_tc_kernel<CG, B_MN, NSTG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem_bytes(NSTG));
+  cudaError_t e = cudaFuncSetAttribute(ns_tc_kernel<CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)TC_SMEM_BYTES);
   if (e != cudaSuccess) { *err = e; return 0; }
   if (CG == 1) {
     cached = n_sms;
@@ -834,38 +999,43 @@ int resident_units(int n_sms, cudaError_t* err) {
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)(n_sms / 2 * 2));
   cfg.blockDim = dim3(TC_THREADS);
-  cfg.dynamicSmemBytes = smem_bytes(NSTG);
+  cfg.dynamicSmemBytes = TC_SMEM_BYTES;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, ns_tc_kernel<CG, B_MN, NSTG>, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&n, ns_tc_kernel<CG>, &cfg);
   if (e != cudaSuccess) { *err = e; return 0; }
   if (n < 1) { *err = cudaErrorLaunchOutOfResources; return 0; }
   cached = n;
   return cached;
 }
 
-template <int CG, bool B_MN, int NSTG>
-cudaError_t launch_one(cudaStream_t st, const Maps5& m, const TcParams& p, int n_sms) {
+template <int CG>
+cudaError_t launch_one(cudaStream_t st, const TcMaps& m, const TcParams& p, int n_sms) {
   cudaError_t e;
-  const int units = resident_units<CG, B_MN, NSTG>(n_sms, &e);
+  const int units = resident_units<CG>(n_sms, &e);
   if (e != cudaSuccess) return e;
-  const int total = p.n_mats * p.n_tiles_per_mat;
-  const int workers = total < units ? total : units;
+  // every worker must be resident for the whole launch (items wait for items of other workers)
+  const int workers = p.total_items < units ? p.total_items : units;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)(workers * CG));
   cfg.blockDim = dim3(TC_THREADS);
-  cfg.dynamicSmemBytes = smem_bytes(NSTG);
+  cfg.dynamicSmemBytes = TC_SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, ns_tc_kernel<CG, B_MN, NSTG>, *m.a, *m.b, *m.c, *m.d, *m.t, p);
+  return cudaLaunchKernelEx(&cfg, ns_tc_kernel<CG>, m, p);
 }
+
+struct BlockTable {
+  TcBlock* dev = nullptr;
+  int n_blocks = 0, total_items = 0;
+};
 
 }  // namespace
 
@@ -873,21 +1043,16 @@ struct TcGroupPlan {
   int64_t s, l, ldx, lds;
   int chunk;
   int cg;                       // CTAs per tile worker (1 or 2)
-  void* X[2];
-  void* A;
-  void* B;
-  // k: K-major operand boxes (64 x 128); mn: MN-major operand boxes (64 x 64: X as the right
-  // operand of the apply, A and B for the blocks read from their mirror image); io: 64 x 32 boxes
-  // for addend loads and result stores
-  CUtensorMap x_k[2], x_mn[2], x_io[2], a_k, a_mn, a_io, b_k, b_mn, b_io;
-  // 4-D forms of the mn maps (both atoms of a slab in one copy); used when the column count is a
-  // multiple of 64 and the driver accepts the layout
-  CUtensorMap x_mn2[2], a_mn2, b_mn2;
+  int group, n_slots;           // matrices per group of the work list, ring slots (2 * group)
+  int ns_steps, cw;
+  TcMaps maps;
   bool wide_x = false, wide_s = false;
   int2* tiles_sym = nullptr;
-  int n_tiles_sym = 0;
+  int n_sym = 0;
   int2* tiles_full = nullptr;
-  int n_tiles_full = 0;
+  int n_full = 0;
+  int* counters = nullptr;
+  std::map<int, BlockTable> tables;   // work list per matrix count
   int n_sms = 148;
 };
 
@@ -900,31 +1065,78 @@ int tc_num_sms() {
   return n;
 }
 
-TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1, int64_t ldx, void* A,
-                            void* B, int64_t lds, char* err, size_t errlen) {
+// Matrices per group of the work list.  Between the tiles of one product of a matrix and the tiles
+// of its next product lie the same product's tiles of the group's other matrices; with about two
+// rounds of the tile workers in between, a worker (and its copies, which run a tile ahead) rarely
+// finds its inputs unfinished.  More matrices per group would only push the intermediates out of L2.
+int tc_group_size(int64_t s, int chunk) {
+  const int cg = (s > 128) ? 2 : 1;
+  const int64_t T = 128 * cg;
+  const int64_t tm = (s + T - 1) / T;
+  const int64_t n_sym = tm * (tm + 1) / 2;
+  const int units = tc_num_sms() / cg;
+  int64_t g = (2 * units + n_sym - 1) / n_sym;
+  if (const char* e = getenv("MULOCO_NS_GROUP")) {     // tuning studies
+    const int v = atoi(e);
+    if (v > 0) g = v;
+  }
+  if (g < 1) g = 1;
+  if (g > chunk) g = chunk;
+  return (int)g;
+}
+
+size_t tc_ring_bytes(int64_t s, int64_t ldx, int64_t lds, int n_slots) {
+  const size_t xb = ((size_t)n_slots * s * ldx * 2 + 1023) / 1024 * 1024;
+  const size_t sb = ((size_t)n_slots * s * lds * 2 + 1023) / 1024 * 1024;
+  return 2 * xb + 2 * sb;
+}
+
+TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, int64_t ldx, void* ring, int64_t lds,
+                            int group, int* counters, int ns_steps, char* err, size_t errlen) {
   TcGroupPlan* pl = new TcGroupPlan();
   pl->s = s; pl->l = l; pl->ldx = ldx; pl->lds = lds; pl->chunk = chunk;
-  pl->X[0] = X0; pl->X[1] = X1; pl->A = A; pl->B = B;
+  pl->group = group; pl->n_slots = 2 * group;
+  pl->ns_steps = ns_steps; pl->cw = 3 * ns_steps;
+  pl->counters = counters;
   pl->n_sms = tc_num_sms();
   pl->cg = (s > 128) ? 2 : 1;
+  const int ns = pl->n_slots;
+  const size_t xb = ((size_t)ns * s * ldx * 2 + 1023) / 1024 * 1024;
+  const size_t sb = ((size_t)ns * s * lds * 2 + 1023) / 1024 * 1024;
+  char* r = reinterpret_cast<char*>(ring);
+  void* XA = r;
+  void* XB = r + xb;
+  void* A = r + 2 * xb;
+  void* B = r + 2 * xb + sb;
+  CUtensorMap* m = pl->maps.m;
   bool ok = true;
-  for (int i = 0; i < 2; ++i) {
-    ok = ok && encode_map(&pl->x_k[i], pl->X[i], l, s, chunk, ldx, BK, 128, true);
-    ok = ok && encode_map(&pl->x_mn[i], pl->X[i], l, s, chunk, ldx, 64, BK, true);
-    ok = ok && encode_map(&pl->x_io[i], pl->X[i], l, s, chunk, ldx, 64, 32, true);
+  ok = ok && encode_map(&m[MAP_X0_K], X0, l, s, chunk, ldx, BK, 128, true);
+  ok = ok && encode_map(&m[MAP_XA_K], XA, l, s, ns, ldx, BK, 128, true);
+  ok = ok && encode_map(&m[MAP_XB_K], XB, l, s, ns, ldx, BK, 128, true);
+  ok = ok && encode_map(&m[MAP_XA_IO], XA, l, s, ns, ldx, 64, 32, true);
+  ok = ok && encode_map(&m[MAP_XB_IO], XB, l, s, ns, ldx, 64, 32, true);
+  ok = ok && encode_map(&m[MAP_A_K], A, s, s, ns, lds, BK, 128, true);
+  ok = ok && encode_map(&m[MAP_A_IO], A, s, s, ns, lds, 64, 32, true);
+  ok = ok && encode_map(&m[MAP_B_K], B, s, s, ns, lds, BK, 128, true);
+  ok = ok && encode_map(&m[MAP_B_IO], B, s, s, ns, lds, 64, 32, true);
+  // MN-major operands: one 4-D copy per slab when the column count is a multiple of 64 and the
+  // driver accepts the layout, else two 64 x 64 boxes
+  pl->wide_x = encode_map_mn2(&m[MAP_X0_MN], X0, l, s, chunk, ldx) && encode_map_mn2(&m[MAP_XA_MN], XA, l, s, ns, ldx) &&
+               encode_map_mn2(&m[MAP_XB_MN], XB, l, s, ns, ldx);
+  if (!pl->wide_x) {
+    ok = ok && encode_map(&m[MAP_X0_MN], X0, l, s, chunk, ldx, 64, BK, true);
+    ok = ok && encode_map(&m[MAP_XA_MN], XA, l, s, ns, ldx, 64, BK, true);
+    ok = ok && encode_map(&m[MAP_XB_MN], XB, l, s, ns, ldx, 64, BK, true);
   }
-  ok = ok && encode_map(&pl->a_k, A, s, s, chunk, lds, BK, 128, true);
-  ok = ok && encode_map(&pl->a_io, A, s, s, chunk, lds, 64, 32, true);
-  ok = ok && encode_map(&pl->a_mn, A, s, s, chunk, lds, 64, BK, true);
-  ok = ok && encode_map(&pl->b_k, B, s, s, chunk, lds, BK, 128, true);
-  ok = ok && encode_map(&pl->b_io, B, s, s, chunk, lds, 64, 32, true);
-  ok = ok && encode_map(&pl->b_mn, B, s, s, chunk, lds, 64, BK, true);
-  pl->wide_x = encode_map_mn2(&pl->x_mn2[0], pl->X[0], l, s, chunk, ldx) &&
-               encode_map_mn2(&pl->x_mn2[1], pl->X[1], l, s, chunk, ldx);
-  pl->wide_s = encode_map_mn2(&pl->a_mn2, A, s, s, chunk, lds) && encode_map_mn2(&pl->b_mn2, B, s, s, chunk, lds);
+  pl->wide_s = encode_map_mn2(&m[MAP_A_MN], A, s, s, ns, lds) && encode_map_mn2(&m[MAP_B_MN], B, s, s, ns, lds);
+  if (!pl->wide_s) {
+    ok = ok && encode_map(&m[MAP_A_MN], A, s, s, ns, lds, 64, BK, true);
+    ok = ok && encode_map(&m[MAP_B_MN], B, s, s, ns, lds, 64, BK, true);
+  }
   if (getenv("MULOCO_VERBOSE"))
-    fprintf(stderr, "muloco: Newton-Schulz plan %lld x %lld, chunk %d: one-copy MN-major slabs for X %s, for A/B %s\n",
-            (long long)s, (long long)l, chunk, pl->wide_x ? "yes" : "no", pl->wide_s ? "yes" : "no");
+    fprintf(stderr, "muloco: Newton-Schulz plan %lld x %lld, chunk %d, groups of %d (ring of %d slots): one-copy "
+            "MN-major slabs for X %s, for A/B %s\n", (long long)s, (long long)l, chunk, group, ns,
+            pl->wide_x ? "yes" : "no", pl->wide_s ? "yes" : "no");
   if (!ok) {
     snprintf(err, errlen, "cuTensorMapEncodeTiled failed for shape %lld x %lld", (long long)s, (long long)l);
     delete pl;
@@ -938,8 +1150,8 @@ TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, void* X1,
   const int tn_full = (int)((l + T - 1) / T);
   for (int tm = 0; tm < tm_n; ++tm)
     for (int tn = 0; tn < tn_full; ++tn) full.push_back(make_int2(tm, tn));
-  pl->n_tiles_sym = (int)sym.size();
-  pl->n_tiles_full = (int)full.size();
+  pl->n_sym = (int)sym.size();
+  pl->n_full = (int)full.size();
   if (cudaMalloc(&pl->tiles_sym, sym.size() * sizeof(int2)) != cudaSuccess ||
       cudaMalloc(&pl->tiles_full, full.size() * sizeof(int2)) != cudaSuccess ||
       cudaMemcpy(pl->tiles_sym, sym.data(), sym.size() * sizeof(int2), cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -955,41 +1167,74 @@ void tc_plan_destroy(TcGroupPlan* pl) {
   if (!pl) return;
   if (pl->tiles_sym) cudaFree(pl->tiles_sym);
   if (pl->tiles_full) cudaFree(pl->tiles_full);
+  for (auto& kv : pl->tables)
+    if (kv.second.dev) cudaFree(kv.second.dev);
   delete pl;
 }
 
-cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int kind, int n_mats, int xin,
-                      const NsIterArgs& args) {
+namespace {
+
+// The work list for the first n_mats matrices of the chunk: groups of `group` matrices, each group
+// product by product (Gram, polynomial, apply of iteration 0, 1, ...), each product matrix by matrix.
+cudaError_t get_table(TcGroupPlan* pl, int n_mats, BlockTable* out) {
+  auto it = pl->tables.find(n_mats);
+  if (it != pl->tables.end()) { *out = it->second; return cudaSuccess; }
+  std::vector<TcBlock> blocks;
+  int64_t item = 0;
+  const int last_ph = pl->cw - 1;
+  for (int g0 = 0; g0 < n_mats; g0 += pl->group) {
+    const int n = (n_mats - g0 < pl->group) ? (n_mats - g0) : pl->group;
+    for (int ph = 0; ph <= last_ph; ++ph) {
+      TcBlock b;
+      memset(&b, 0, sizeof b);
+      b.kind = (ph % 3 == 0) ? GEMM_GRAM : (ph % 3 == 1) ? GEMM_POLY : (ph == last_ph ? GEMM_FINAL : GEMM_APPLY);
+      b.ph = ph;
+      b.mat0 = g0; b.n_mats = n;
+      b.first_item = (int)item;
+      b.n_items = n * ((ph % 3 == 2) ? pl->n_full : pl->n_sym);
+      item += b.n_items;
+      blocks.push_back(b);
+    }
+  }
+  if (item >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  BlockTable t;
+  t.n_blocks = (int)blocks.size();
+  t.total_items = (int)item;
+  cudaError_t e = cudaMalloc(&t.dev, blocks.size() * sizeof(TcBlock));
+  if (e != cudaSuccess) return e;
+  e = cudaMemcpy(t.dev, blocks.data(), blocks.size() * sizeof(TcBlock), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) { cudaFree(t.dev); return e; }
+  pl->tables[n_mats] = t;
+  *out = t;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int n_mats, const NsIterArgs& args) {
   if (n_mats <= 0) return cudaSuccess;
+  if (n_mats > pl->chunk) return cudaErrorInvalidValue;
+  BlockTable t;
+  cudaError_t e = get_table(pl, n_mats, &t);
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(pl->counters, 0, (size_t)n_mats * pl->cw * sizeof(int), st);
+  if (e != cudaSuccess) return e;
   TcParams p;
   memset(&p, 0, sizeof(p));
-  p.kind = kind; p.n_mats = n_mats;
+  p.blocks = t.dev; p.n_blocks = t.n_blocks; p.total_items = t.total_items;
+  p.tiles_sym = pl->tiles_sym; p.tiles_full = pl->tiles_full;
+  p.n_sym = pl->n_sym; p.n_full = pl->n_full;
+  p.s = (int)pl->s; p.l = (int)pl->l;
+  p.last_ph = pl->cw - 1;
   p.a = args.a; p.b = args.b; p.c = args.c;
   p.scales = args.scales; p.mats = args.mats; p.sink_mode = args.sink_mode;
-  p.s = pl->s; p.l = pl->l; p.status = args.status;
-  p.M = (int)pl->s;
-  Maps5 m;
-  if (kind == GEMM_GRAM) {
-    p.N = (int)pl->s; p.Kd = (int)pl->l; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
-    m = Maps5{&pl->x_k[xin], &pl->x_k[xin], &pl->a_io, &pl->a_io, &pl->a_mn};
-    return pl->cg == 2 ? launch_one<2, false, 5>(st, m, p, pl->n_sms) : launch_one<1, false, 5>(st, m, p, pl->n_sms);
-  }
-  if (kind == GEMM_POLY) {
-    p.N = (int)pl->s; p.Kd = (int)pl->s; p.tiles = pl->tiles_sym; p.n_tiles_per_mat = pl->n_tiles_sym;
-    p.a_tri = 1; p.b_tri = 1;
-    p.s_wide = pl->wide_s;
-    m = Maps5{&pl->a_k, &pl->a_k, &pl->a_io, &pl->b_io, pl->wide_s ? &pl->a_mn2 : &pl->a_mn};
-    return pl->cg == 2 ? launch_one<2, false, 5>(st, m, p, pl->n_sms) : launch_one<1, false, 5>(st, m, p, pl->n_sms);
-  }
-  p.N = (int)pl->l; p.Kd = (int)pl->s; p.tiles = pl->tiles_full; p.n_tiles_per_mat = pl->n_tiles_full;
-  // FINAL stores nothing through tmD; the map still has to be a valid one
-  p.a_tri = 1;      // the left operand is the polynomial B, stored on and above the diagonal
-  p.b_wide = pl->wide_x; p.s_wide = pl->wide_s;
-  m = Maps5{&pl->b_k, pl->wide_x ? &pl->x_mn2[xin] : &pl->x_mn[xin], &pl->x_io[xin], &pl->x_io[1 - xin],
-            pl->wide_s ? &pl->b_mn2 : &pl->b_mn};
-  if (kind == GEMM_APPLY)
-    return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
-  return pl->cg == 2 ? launch_one<2, true, 5>(st, m, p, pl->n_sms) : launch_one<1, true, 5>(st, m, p, pl->n_sms);
+  p.x_wide = pl->wide_x; p.s_wide = pl->wide_s;
+  p.n_slots = pl->n_slots;
+  p.counters = pl->counters; p.cw = pl->cw;
+  p.status = args.status;
+  p.wait_limit_ns = args.wait_limit_ns ? args.wait_limit_ns : 2000000000ull;
+  p.debug_withhold = args.debug_withhold;
+  return pl->cg == 2 ? launch_one<2>(st, pl->maps, p, pl->n_sms) : launch_one<1>(st, pl->maps, p, pl->n_sms);
 }
 
 }  // namespace muloco

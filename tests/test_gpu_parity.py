@@ -600,6 +600,43 @@ def test_nonfinite_gradient_of_an_adamw_tensor_is_reported(grad_dtype):
 
 
 # ---------------------------------------------------------------------------
+# failure path of the tensor-core kernel: a wait that runs out (nothing faults, nothing hangs)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("batch,m,n", [(1, 256, 256), (1, 128, 128), (40, 512, 768), (3, 64, 200)])
+def test_bounded_wait_runs_out_and_the_context_stays_usable(batch, m, n):
+    """One operand copy of the first tile is withheld, so the waits that depend on it (the MMA
+    issuer's, the epilogue's, then the other CTAs' waits for that tile's result) run out after
+    the 2 ms the test sets: the kernel returns, MULOCO_ETIMEOUT is reported once, and the same
+    context then computes a correct Newton-Schulz result."""
+    import time
+    import torch
+    from paper_2505_23725_b200 import binding
+    w = configs.Workload("ns-only", K=1, H=1, J=1, tensors=[], muon_lr=0.02, muon_beta=0.95, muon_wd=0.0,
+                         outer_lr=1.0, outer_momentum=0.0)
+    ctx = gpu_for(w, [])
+    rng = np.random.default_rng(77)
+    X = np.stack([synth.lowrank_plus_noise(rng, m, n) for _ in range(batch)])
+    Xd = torch.from_numpy(X).cuda()
+    ctx.newton_schulz(Xd, ns_mode="bf16")                  # builds the plan; a normal call first
+    ctx.sync_status()
+    ctx.debug_set(binding.DEBUG_WAIT_LIMIT_NS, 2_000_000)
+    ctx.debug_set(binding.DEBUG_WITHHOLD_COPY, 1)
+    t0 = time.perf_counter()
+    ctx.newton_schulz(Xd, ns_mode="bf16")
+    with pytest.raises(binding.MulocoError) as e:
+        ctx.sync_status()
+    assert e.value.status == binding.ETIMEOUT
+    assert time.perf_counter() - t0 < 5.0                   # it gave up after milliseconds, not at a watchdog
+    ctx.sync_status()                                       # the flag is cleared once read
+    ctx.debug_set(binding.DEBUG_WAIT_LIMIT_NS, 0)           # back to the default limit
+    out = _np(ctx.newton_schulz(Xd, ns_mode="bf16"))        # the switch was one-shot: this call is whole
+    ctx.sync_status()
+    for b in range(batch):
+        assert relfro(out[b], O.newton_schulz(X[b])) < 2e-2
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------
 # bf16 sources: every access shape of the staging kernel (wide and tall tensors, aligned and not)
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("m,n", [(384, 256), (96, 1032), (96, 1031), (130, 96), (257, 131), (132, 514), (1024, 64),
