@@ -306,10 +306,13 @@ outer_sync2_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* _
 // Row-wise quantisation (one absmax block per row; Section 6.3 and the row-wise panels of the
 // quantisation ablation): one CTA per row.  The row's pseudogradient (or, with two stages, the mean
 // of the workers' dequantised deltas) is staged in shared memory between the pass that finds the
-// row's absmax and the pass that quantises it.  With two stages every replica is read twice: once
-// for its own absmax, once to be quantised with it.  Arithmetic and order are those of the block
-// kernels, so codes are bit-exact against the same reference.
+// row's absmax and the pass that quantises it.  With two stages a worker's row is needed twice (for
+// its absmax, then to be quantised with it): outer_sync_row1_kernel stages it in shared memory
+// beside the running sum, so every replica (and error-feedback accumulator) is read from memory
+// once; rows too long for two staged copies take outer_sync_row_kernel, which reads them twice.
+// Arithmetic and order are those of the block kernels, so codes are bit-exact against the same reference.
 constexpr int ROW_THREADS = 256;
+constexpr int ROW_PIECES = 4;            // pieces of four columns a thread can hold in registers
 
 __device__ __forceinline__ float block_max(float v, float* red) {
   v = warp_max(v);
@@ -332,6 +335,210 @@ __device__ __forceinline__ float quant_dequant1(float x, float amax, bool& bad) 
   float r = rintf(__fmul_rn(x, inv));
   r = fminf(fmaxf(r, -qmax), qmax);
   return __fmul_rn(r, scale);
+}
+
+// Two quantisations per sync, every array read once.  Shared memory: xbuf[cols4] (the current
+// worker's delta, or its error-feedback sum) and acc[cols4] (running sum of what the workers sent);
+// every thread only ever touches the entries of its own columns, so the two arrays need no barrier
+// of their own.  Pieces of four columns per thread (16-byte accesses when the row allows it).
+// Rows of up to ROW_PIECES * ROW_THREADS pieces (4096 columns) run software-pipelined: theta stays
+// in registers for the whole row, and the next worker's replica (and accumulator) is already on
+// its way while the current worker's absmax is reduced over the CTA.
+template <int QB, bool EF>
+__global__ void __launch_bounds__(ROW_THREADS)
+outer_sync_row1_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps,
+                       float* const* __restrict__ efs, int K, int64_t n_rows, int64_t cols_pad, float eta,
+                       float mu, float inv_k, float ef_beta, int* __restrict__ status) {
+  extern __shared__ float rowbuf[];      // [cols_pad] xbuf, [cols_pad] acc
+  __shared__ float red[ROW_THREADS / 32];
+  __shared__ int vec_ok;
+  const int64_t unit = blockIdx.x;
+  if (unit >= n_rows) return;
+  const int seg = find_seg(segs, n_segs, unit);
+  const SyncSeg s = segs[seg];
+  const int64_t row = unit - s.unit_begin;
+  const int64_t cols = s.cols;
+  const int64_t off0 = row * cols;
+  float* const* rp = reps + s.rep_index;
+  float* const* ep = EF ? efs + s.rep_index : nullptr;
+  float* xbuf = rowbuf;
+  float* accb = rowbuf + cols_pad;
+  bool bad = false;
+  float* tgp = s.theta_g + off0;
+  float* up = s.u + off0;
+  if (threadIdx.x == 0) {
+    uintptr_t bits = (uintptr_t)tgp | (uintptr_t)up;
+    for (int k = 0; k < K; ++k) {
+      bits |= (uintptr_t)(rp[k] + off0);
+      if (EF) bits |= (uintptr_t)(ep[k] + off0);
+    }
+    vec_ok = ((bits & 15) == 0) ? 1 : 0;
+  }
+  __syncthreads();
+  const bool vec = vec_ok != 0;
+  const int64_t n4 = (cols + 3) >> 2;    // pieces of four columns; the last one may be short
+  auto nvalid_of = [&](int64_t c) { return (cols - c >= 4) ? 4 : (int)(cols - c); };
+  auto load_theta = [&](int64_t c, bool v4, int nvalid, float (&t)[4]) {
+    if (v4) {
+      const float4 tt = *reinterpret_cast<const float4*>(tgp + c);
+      t[0] = tt.x; t[1] = tt.y; t[2] = tt.z; t[3] = tt.w;
+    } else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) t[q] = (q < nvalid) ? tgp[c + q] : 0.f;
+    }
+  };
+
+  for (int64_t i = threadIdx.x; i < n4; i += ROW_THREADS)
+    *reinterpret_cast<float4*>(accb + 4 * i) = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  if (n4 <= (int64_t)ROW_PIECES * ROW_THREADS) {
+    // ---- pipelined: this thread's pieces are i = threadIdx.x + j * ROW_THREADS, j < ROW_PIECES ----
+    float t[ROW_PIECES][4], rv[ROW_PIECES][4], ev[ROW_PIECES][4];
+    auto fetch = [&](int k) {
+#pragma unroll
+      for (int j = 0; j < ROW_PIECES; ++j) {
+        const int64_t i = threadIdx.x + (int64_t)j * ROW_THREADS;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { rv[j][q] = 0.f; ev[j][q] = 0.f; }
+        if (i < n4) {
+          const int64_t c = 4 * i;
+          const int nvalid = nvalid_of(c);
+          const bool v4 = vec && nvalid == 4;
+          load4(rp[k] + off0 + c, v4, nvalid, rv[j]);
+          if (EF) load4(ep[k] + off0 + c, v4, nvalid, ev[j]);
+        }
+      }
+    };
+#pragma unroll
+    for (int j = 0; j < ROW_PIECES; ++j) {
+      const int64_t i = threadIdx.x + (int64_t)j * ROW_THREADS;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) t[j][q] = 0.f;
+      if (i < n4) load_theta(4 * i, vec && nvalid_of(4 * i) == 4, nvalid_of(4 * i), t[j]);
+    }
+    fetch(0);
+    for (int k = 0; k < K; ++k) {
+      float lm = 0.f;
+#pragma unroll
+      for (int j = 0; j < ROW_PIECES; ++j) {
+        const int64_t i = threadIdx.x + (int64_t)j * ROW_THREADS;
+        if (i < n4) {
+          const int64_t c = 4 * i;
+          const int nvalid = nvalid_of(c);
+          float x[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float d = __fsub_rn(t[j][q], rv[j][q]);
+            x[q] = EF ? __fadd_rn(__fmul_rn(ef_beta, ev[j][q]), d) : d;
+            if (q >= nvalid) x[q] = 0.f;
+            const float a = fabsf(x[q]);
+            if (!(a <= FLT_MAX)) bad = true;
+            lm = fmaxf(lm, a);
+          }
+          *reinterpret_cast<float4*>(xbuf + c) = make_float4(x[0], x[1], x[2], x[3]);
+        }
+      }
+      if (k + 1 < K) fetch(k + 1);       // in flight during the reduction and the quantising pass
+      const float amax = block_max(lm, red);
+#pragma unroll
+      for (int j = 0; j < ROW_PIECES; ++j) {
+        const int64_t i = threadIdx.x + (int64_t)j * ROW_THREADS;
+        if (i < n4) {
+          const int64_t c = 4 * i;
+          const int nvalid = nvalid_of(c);
+          const bool v4 = vec && nvalid == 4;
+          const float4 xv = *reinterpret_cast<const float4*>(xbuf + c);
+          float4 av = *reinterpret_cast<const float4*>(accb + c);
+          const float x[4] = {xv.x, xv.y, xv.z, xv.w};
+          float sent[4], en[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            sent[q] = quant_dequant1<QB>(x[q], amax, bad);
+            en[q] = __fsub_rn(x[q], sent[q]);
+          }
+          if (EF) store4(ep[k] + off0 + c, v4, nvalid, en);
+          av.x = __fadd_rn(av.x, sent[0]); av.y = __fadd_rn(av.y, sent[1]);
+          av.z = __fadd_rn(av.z, sent[2]); av.w = __fadd_rn(av.w, sent[3]);
+          *reinterpret_cast<float4*>(accb + c) = av;
+        }
+      }
+    }
+  } else {
+    for (int k = 0; k < K; ++k) {
+      float* r = rp[k] + off0;
+      float* e = EF ? ep[k] + off0 : nullptr;
+      float lm = 0.f;
+      for (int64_t i = threadIdx.x; i < n4; i += ROW_THREADS) {
+        const int64_t c = 4 * i;
+        const int nvalid = nvalid_of(c);
+        const bool v4 = vec && nvalid == 4;
+        float t[4], rv[4], ev[4] = {0.f, 0.f, 0.f, 0.f}, x[4];
+        load_theta(c, v4, nvalid, t);                     // read K times: a cache hit after the first
+        load4(r + c, v4, nvalid, rv);
+        if (EF) load4(e + c, v4, nvalid, ev);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float d = __fsub_rn(t[q], rv[q]);
+          x[q] = EF ? __fadd_rn(__fmul_rn(ef_beta, ev[q]), d) : d;
+          if (q >= nvalid) x[q] = 0.f;
+          const float a = fabsf(x[q]);
+          if (!(a <= FLT_MAX)) bad = true;
+          lm = fmaxf(lm, a);
+        }
+        *reinterpret_cast<float4*>(xbuf + c) = make_float4(x[0], x[1], x[2], x[3]);
+      }
+      const float amax = block_max(lm, red);
+      for (int64_t i = threadIdx.x; i < n4; i += ROW_THREADS) {
+        const int64_t c = 4 * i;
+        const int nvalid = nvalid_of(c);
+        const bool v4 = vec && nvalid == 4;
+        const float4 xv = *reinterpret_cast<const float4*>(xbuf + c);
+        float4 av = *reinterpret_cast<const float4*>(accb + c);
+        const float x[4] = {xv.x, xv.y, xv.z, xv.w};
+        float sent[4], en[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          sent[q] = quant_dequant1<QB>(x[q], amax, bad);
+          en[q] = __fsub_rn(x[q], sent[q]);
+        }
+        if (EF) store4(e + c, v4, nvalid, en);
+        av.x = __fadd_rn(av.x, sent[0]); av.y = __fadd_rn(av.y, sent[1]);
+        av.z = __fadd_rn(av.z, sent[2]); av.w = __fadd_rn(av.w, sent[3]);
+        *reinterpret_cast<float4*>(accb + c) = av;
+      }
+    }
+  }
+  // the mean, its absmax, the second quantisation, the outer step, the broadcast
+  float lm = 0.f;
+  for (int64_t i = threadIdx.x; i < n4; i += ROW_THREADS) {
+    float4 av = *reinterpret_cast<const float4*>(accb + 4 * i);
+    av.x = __fmul_rn(av.x, inv_k); av.y = __fmul_rn(av.y, inv_k);
+    av.z = __fmul_rn(av.z, inv_k); av.w = __fmul_rn(av.w, inv_k);
+    *reinterpret_cast<float4*>(accb + 4 * i) = av;
+    lm = fmaxf(fmaxf(lm, fabsf(av.x)), fmaxf(fabsf(av.y), fmaxf(fabsf(av.z), fabsf(av.w))));
+  }
+  const float amax = block_max(lm, red);
+  for (int64_t i = threadIdx.x; i < n4; i += ROW_THREADS) {
+    const int64_t c = 4 * i;
+    const int nvalid = nvalid_of(c);
+    const bool v4 = vec && nvalid == 4;
+    const float4 av = *reinterpret_cast<const float4*>(accb + c);
+    const float m4[4] = {av.x, av.y, av.z, av.w};
+    float t[4], uu[4], un[4], tn[4];
+    load_theta(c, v4, nvalid, t);
+    load4(up + c, v4, nvalid, uu);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float psi = quant_dequant1<QB>(m4[q], amax, bad);
+      const float epq = eta * psi;
+      un[q] = fmaf(mu, uu[q], epq);
+      tn[q] = t[q] - fmaf(mu, un[q], epq);
+    }
+    store4(up + c, v4, nvalid, un);
+    store4(tgp + c, v4, nvalid, tn);
+    for (int k = 0; k < K; ++k) store4(rp[k] + off0 + c, v4, nvalid, tn);
+  }
+  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, ST_NONFINITE);
 }
 
 template <int QB, bool TWO, bool EF>
@@ -536,6 +743,10 @@ cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_s
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   const float inv_k = 1.0f / (float)K;
   const bool two = (stages == 2);
+  // two stages: two staged copies of the row (the worker's values and the running sum) when they fit
+  const int64_t cols_pad = (max_cols + 3) / 4 * 4;
+  const size_t smem1 = 2 * (size_t)cols_pad * sizeof(float);
+  const bool single_read = two && smem1 <= 200 * 1024;
 #define MULOCO_ROW_LAUNCH(QB, TWO, EF)                                                                   \
   do {                                                                                                   \
     cudaError_t e_ = cudaFuncSetAttribute(outer_sync_row_kernel<QB, TWO, EF>,                            \
@@ -544,9 +755,19 @@ cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_s
     outer_sync_row_kernel<QB, TWO, EF><<<(unsigned)n_rows, ROW_THREADS, smem, st>>>(                     \
         segs, n_segs, replicas, ef, K, n_rows, outer_lr, mu, inv_k, ef_beta, status);                    \
   } while (0)
+#define MULOCO_ROW1_LAUNCH(QB, EF)                                                                       \
+  do {                                                                                                   \
+    cudaError_t e_ = cudaFuncSetAttribute(outer_sync_row1_kernel<QB, EF>,                                \
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024)); \
+    if (e_ != cudaSuccess) return e_;                                                                    \
+    outer_sync_row1_kernel<QB, EF><<<(unsigned)n_rows, ROW_THREADS, smem1, st>>>(                        \
+        segs, n_segs, replicas, ef, K, n_rows, cols_pad, outer_lr, mu, inv_k, ef_beta, status);          \
+  } while (0)
 #define MULOCO_ROW_BITS(QB)                                   \
   do {                                                        \
-    if (two && ef) MULOCO_ROW_LAUNCH(QB, true, true);         \
+    if (single_read && ef) MULOCO_ROW1_LAUNCH(QB, true);      \
+    else if (single_read) MULOCO_ROW1_LAUNCH(QB, false);      \
+    else if (two && ef) MULOCO_ROW_LAUNCH(QB, true, true);    \
     else if (two) MULOCO_ROW_LAUNCH(QB, true, false);         \
     else MULOCO_ROW_LAUNCH(QB, false, false);                 \
   } while (0)
@@ -554,6 +775,7 @@ cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_s
   else if (quant_bits == 4) MULOCO_ROW_BITS(4);
   else MULOCO_ROW_BITS(2);
 #undef MULOCO_ROW_BITS
+#undef MULOCO_ROW1_LAUNCH
 #undef MULOCO_ROW_LAUNCH
   return cudaGetLastError();
 }
