@@ -295,9 +295,25 @@ MULOCO_API muloco_status muloco_get_timings(muloco_ctx* ctx, float* ms, int64_t*
  * parameters theta_k of some of its (worker, matrix) pairs have been updated, or partly
  * updated, and others not, and nothing records which.  A caller that wants to continue
  * restores theta_k and the momenta of that step from its own copy (a checkpoint of the
- * caller-owned tensors plus muloco_get_state / muloco_set_state) and repeats the step. */
-enum { MULOCO_DEBUG_WAIT_LIMIT_NS = 1, MULOCO_DEBUG_WITHHOLD_COPY = 2 };
+ * caller-owned tensors plus muloco_get_state / muloco_set_state) and repeats the step.
+ *
+ * Workspace canaries (the library's stand-in for a memory checker): every region of the
+ * Newton-Schulz workspace (staged input, ring of intermediates, norm partials, scales, tile
+ * counters) lies between guard zones whose adjoining 64 bytes hold a fixed pattern.
+ *   MULOCO_DEBUG_CANARIES : value != 0 makes every Newton-Schulz chunk write the canaries
+ *       before it runs and compare them after (this waits for the stream after every chunk: a
+ *       debugging mode).  muloco_check_workspace reports the first canary found overwritten
+ *       since its last call (MULOCO_ESTATE, text in muloco_last_error), else MULOCO_OK.
+ *   MULOCO_DEBUG_CORRUPT_CANARY : test hook; value = index of a workspace region whose canary
+ *       the host overwrites (one byte, by a memset on the stream) in the next chunk, so that
+ *       the check has something to find.  One-shot.
+ * A debug build of the library (-DMULOCO_DEBUG, build.build_library(debug=True)) adds
+ * device-side checks of the indices the kernels derive; a failed check raises a flag that
+ * muloco_sync_status reports as MULOCO_ECUDA ("out-of-range index"), and the access is skipped. */
+enum { MULOCO_DEBUG_WAIT_LIMIT_NS = 1, MULOCO_DEBUG_WITHHOLD_COPY = 2, MULOCO_DEBUG_CANARIES = 3,
+       MULOCO_DEBUG_CORRUPT_CANARY = 4 };
 MULOCO_API muloco_status muloco_debug_set(muloco_ctx* ctx, int32_t what, int64_t value);
+MULOCO_API muloco_status muloco_check_workspace(muloco_ctx* ctx);
 
 /* Waits for the stream and returns the device status word as a muloco_status
  * (MULOCO_OK, MULOCO_ENONFINITE, MULOCO_ETIMEOUT, MULOCO_ECUDA); clears it. */

@@ -25,7 +25,7 @@ STATUS_NAMES = ["OK", "EINVAL", "ESHAPE", "ENOMEM", "ECUDA", "ENONFINITE", "ETIM
 MUON, ADAMW = 0, 1
 NS_BF16, NS_FP32 = 0, 1
 F32, BF16 = 0, 1
-DEBUG_WAIT_LIMIT_NS, DEBUG_WITHHOLD_COPY = 1, 2
+DEBUG_WAIT_LIMIT_NS, DEBUG_WITHHOLD_COPY, DEBUG_CANARIES, DEBUG_CORRUPT_CANARY = 1, 2, 3, 4
 PHASES = ["prologue", "ns", "adamw", "sync", "copy"]
 
 EXPORTS = [
@@ -33,7 +33,7 @@ EXPORTS = [
     "muloco_outer_sync", "muloco_outer_sync_host", "muloco_fragments_due", "muloco_newton_schulz",
     "muloco_quantize", "muloco_topk_sparsify", "muloco_pseudogradient", "muloco_get_state", "muloco_set_state",
     "muloco_set_timing", "muloco_get_timings", "muloco_sync_status", "muloco_last_error",
-    "muloco_newton_schulz_static", "muloco_debug_set",
+    "muloco_newton_schulz_static", "muloco_debug_set", "muloco_check_workspace",
 ]
 
 
@@ -103,6 +103,7 @@ def load_library():
     lib.muloco_last_error.argtypes = [vp]
     lib.muloco_last_error.restype = C.c_char_p
     lib.muloco_debug_set.argtypes = [vp, i32, i64]
+    lib.muloco_check_workspace.argtypes = [vp]
     lib.muloco_newton_schulz_static.argtypes = [vp, vp, i32, i64, i64, vp, C.c_char_p, C.c_size_t]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -400,6 +401,10 @@ class MuLoCo:
 
     def sync_status(self):
         self._check(self.lib.muloco_sync_status(self.ctx))
+
+    def check_workspace(self):
+        """muloco_check_workspace: raises MulocoError(ESTATE) if a workspace canary was overwritten."""
+        self._check(self.lib.muloco_check_workspace(self.ctx))
 
     def debug_set(self, what: int, value: int):
         """muloco_debug_set (test hooks of the failure path)."""

@@ -9,6 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmuloco.so")
+LIB_DEBUG = os.path.join(HERE, "libmuloco_debug.so")   # the same sources with -DMULOCO_DEBUG (index checks in the kernels)
 SOURCES = ["capi.cu", "elementwise.cu", "outer_sync.cu", "topk.cu", "ns_fp32.cu", "ns_tc.cu", "ns_static.cu"]
 
 
@@ -19,24 +20,31 @@ def _nvcc() -> str:
     return cand
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(lib_path: str = LIB) -> bool:
+    if not os.path.exists(lib_path):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib_path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "muloco.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False, lib_path: str = LIB) -> str:
-    """Compile every CUDA source of the package for sm_100a into one shared library."""
-    if not force and lib_path == LIB and not needs_build():
-        return LIB
+def build_library(force: bool = False, verbose: bool = False, lib_path: str = None, debug: bool = False) -> str:
+    """Compile every CUDA source of the package for sm_100a into one shared library.
+    debug=True builds libmuloco_debug.so: the same sources with -DMULOCO_DEBUG, i.e. with the
+    kernels' index checks compiled in (a failed check raises a status flag, nothing traps)."""
+    if lib_path is None:
+        lib_path = LIB_DEBUG if debug else LIB
+    if not force and lib_path in (LIB, LIB_DEBUG) and not needs_build(lib_path):
+        return lib_path
     objs = []
-    bdir = os.path.join(HERE, "_build") if lib_path == LIB else lib_path + ".objs"
+    bdir = os.path.join(HERE, "_build") if lib_path == LIB else (
+        os.path.join(HERE, "_build", "debug") if lib_path == LIB_DEBUG else lib_path + ".objs")
     os.makedirs(bdir, exist_ok=True)
     common = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
+    if debug:
+        common += ["-DMULOCO_DEBUG"]
     if verbose:
         common += ["-Xptxas", "-v"]
     common += os.environ.get("MULOCO_NVCC_FLAGS", "").split()   # extra -D... for tuning studies

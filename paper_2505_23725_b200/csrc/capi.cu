@@ -30,10 +30,15 @@ struct TensorInfo {
   int64_t numel() const { return rows * cols; }
 };
 
+struct WsRegion { const char* name; size_t off, bytes; };
+
 struct WsLayout {   // byte offsets inside the workspace for one shape group
   // fp32 engine: x0, x1, a, b are chunk-sized.  bf16 engine: x0 is the chunk-sized staged input and
   // `ring` holds the intermediates of 2 * group matrices; `counters` counts finished tiles.
-  size_t x0, x1, a, b, ring, partials, scales, counters, total;
+  // Every region lies between guard zones of at least 1 KB; the 64 bytes right before and right
+  // after a region are its canaries (see muloco_check_workspace).
+  size_t x0 = 0, x1 = 0, a = 0, b = 0, ring = 0, partials = 0, scales = 0, counters = 0, total = 0;
+  std::vector<WsRegion> regions;
 };
 
 struct Group {
@@ -79,25 +84,34 @@ int engine_for(int requested_mode, int64_t s) {
   return (requested_mode == MULOCO_NS_BF16 && s >= BF16_MIN_S) ? MULOCO_NS_BF16 : MULOCO_NS_FP32;
 }
 
+constexpr size_t WS_GUARD = 1024, WS_CANARY = 64;
+constexpr int WS_CANARY_BYTE = 0xC5;
+
 WsLayout make_layout(int64_t s, int64_t ldx, int64_t lds, int chunk, int n_part, int elt, int ring_group,
                      int ns_steps) {
   WsLayout w;
-  memset(&w, 0, sizeof w);
   size_t off = 0;
-  const size_t xb = align_up((size_t)chunk * s * ldx * elt, 1024);
-  w.x0 = off; off += xb;
+  auto place = [&](const char* name, size_t bytes) {
+    off = align_up(off + WS_GUARD, 1024);
+    w.regions.push_back(WsRegion{name, off, bytes});
+    const size_t at = off;
+    off += bytes;
+    return at;
+  };
+  const size_t xb = (size_t)chunk * s * ldx * elt;
+  w.x0 = place("X0", xb);
   if (elt == 2) {
-    w.ring = off; off += tc_ring_bytes(s, ldx, lds, 2 * ring_group);
+    w.ring = place("ring", tc_ring_bytes(s, ldx, lds, 2 * ring_group));
   } else {
-    const size_t sb = align_up((size_t)chunk * s * lds * elt, 1024);
-    w.x1 = off; off += xb;
-    w.a = off; off += sb;
-    w.b = off; off += sb;
+    const size_t sb = (size_t)chunk * s * lds * elt;
+    w.x1 = place("X1", xb);
+    w.a = place("A", sb);
+    w.b = place("B", sb);
   }
-  w.partials = off; off += align_up((size_t)chunk * n_part * sizeof(float), 1024);
-  w.scales = off; off += align_up((size_t)chunk * sizeof(float2), 1024);
-  w.counters = off; off += align_up((size_t)chunk * 3 * ns_steps * sizeof(int), 1024);
-  w.total = off;
+  w.partials = place("partials", (size_t)chunk * n_part * sizeof(float));
+  w.scales = place("scales", (size_t)chunk * sizeof(float2));
+  w.counters = place("counters", (size_t)chunk * 3 * ns_steps * sizeof(int));
+  w.total = align_up(off + WS_GUARD, 1024);
   return w;
 }
 
@@ -140,6 +154,9 @@ struct muloco_ctx {
   int* d_status = nullptr;
   unsigned long long wait_limit_ns = 0;   // limit of the device-side waits of the bf16 engine (0: its default)
   int debug_withhold = 0;                 // test hook, see muloco_debug_set
+  bool canaries = false;                  // write and verify the workspace canaries around every chunk
+  int corrupt_region = -1;                // test hook: one canary byte of this region is overwritten (one-shot)
+  std::string canary_report;              // first violation since the last muloco_check_workspace
 
   std::vector<int> muon_ids, adam_ids;
   std::vector<Group> groups;
@@ -294,6 +311,44 @@ muloco_status setup_group(muloco_ctx* c, Group& g, char* ws, int mode) {
   return MULOCO_OK;
 }
 
+// Canaries of a group's layout inside workspace `ws`: written before a chunk runs ...
+muloco_status write_canaries(muloco_ctx* c, const Group& g, char* ws) {
+  for (const WsRegion& r : g.ws.regions) {
+    CK(cudaMemsetAsync(ws + r.off - WS_CANARY, WS_CANARY_BYTE, WS_CANARY, c->st));
+    CK(cudaMemsetAsync(ws + r.off + r.bytes, WS_CANARY_BYTE, WS_CANARY, c->st));
+  }
+  if (c->corrupt_region >= 0 && c->corrupt_region < (int)g.ws.regions.size()) {
+    // test hook: a host-initiated memset stands in for a kernel that wrote past a region's end
+    const WsRegion& r = g.ws.regions[c->corrupt_region];
+    CK(cudaMemsetAsync(ws + r.off + r.bytes + 3, 0, 1, c->st));
+  }
+  c->corrupt_region = -1;
+  return MULOCO_OK;
+}
+
+// ... and verified after it has run (waits for the stream).
+muloco_status verify_canaries(muloco_ctx* c, const Group& g, char* ws) {
+  const size_t n = g.ws.regions.size();
+  std::vector<unsigned char> h(2 * n * WS_CANARY);
+  for (size_t i = 0; i < n; ++i) {
+    const WsRegion& r = g.ws.regions[i];
+    CK(cudaMemcpyAsync(h.data() + (2 * i) * WS_CANARY, ws + r.off - WS_CANARY, WS_CANARY, cudaMemcpyDeviceToHost, c->st));
+    CK(cudaMemcpyAsync(h.data() + (2 * i + 1) * WS_CANARY, ws + r.off + r.bytes, WS_CANARY, cudaMemcpyDeviceToHost, c->st));
+  }
+  CK(cudaStreamSynchronize(c->st));
+  for (size_t i = 0; i < n && c->canary_report.empty(); ++i)
+    for (int side = 0; side < 2 && c->canary_report.empty(); ++side)
+      for (size_t b = 0; b < WS_CANARY; ++b)
+        if (h[(2 * i + side) * WS_CANARY + b] != WS_CANARY_BYTE) {
+          char buf[256];
+          snprintf(buf, sizeof buf, "workspace canary %s region '%s' (shape group %lld x %lld) was overwritten at byte %zu",
+                   side ? "after" : "before", g.ws.regions[i].name, (long long)g.s, (long long)g.l, b);
+          c->canary_report = buf;
+          break;
+        }
+  return MULOCO_OK;
+}
+
 // One chunk of matrices through prologue + Newton-Schulz + sink.
 muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_mats, int n_mats,
                            int mode, int src_mode, int sink_mode, int g_is_bf16) {
@@ -301,6 +356,10 @@ muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_m
   float* partials = reinterpret_cast<float*>(ws + g.ws.partials);
   float2* scales = reinterpret_cast<float2*>(ws + g.ws.scales);
   void* X[2] = {ws + g.ws.x0, ws + g.ws.x1};
+  if (c->canaries) {
+    const muloco_status cs = write_canaries(c, g, ws);
+    if (cs != MULOCO_OK) return cs;
+  }
   {
     PhaseTimer t(c, MULOCO_PH_PROLOGUE);
     launch_prologue(c->st, d_mats, n_mats, g.s, g.l, src_mode, g_is_bf16, f.muon_beta, f.muon_nesterov,
@@ -321,7 +380,7 @@ muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_m
     CK(tc_launch(c->st, g.plan, n_mats, a));
     c->launches += 1;
     CK(cudaGetLastError());
-    return MULOCO_OK;
+    return c->canaries ? verify_canaries(c, g, ws) : MULOCO_OK;
   }
   for (int it = 0; it < f.ns_steps; ++it) {
     const int xin = it & 1;
@@ -340,7 +399,7 @@ muloco_status run_ns_chunk(muloco_ctx* c, Group& g, char* ws, const MatDesc* d_m
     c->launches += 3;
   }
   CK(cudaGetLastError());
-  return MULOCO_OK;
+  return c->canaries ? verify_canaries(c, g, ws) : MULOCO_OK;
 }
 
 muloco_status build_sync_tables(muloco_ctx* c) {
@@ -1072,7 +1131,23 @@ MULOCO_API muloco_status muloco_debug_set(muloco_ctx* c, int32_t what, int64_t v
     c->debug_withhold = value != 0;
     return MULOCO_OK;
   }
+  if (what == MULOCO_DEBUG_CANARIES) {
+    c->canaries = value != 0;
+    return MULOCO_OK;
+  }
+  if (what == MULOCO_DEBUG_CORRUPT_CANARY) {
+    c->corrupt_region = (int)value;
+    return MULOCO_OK;
+  }
   return fail(c, MULOCO_EINVAL, "unknown debug switch %d", what);
+}
+
+MULOCO_API muloco_status muloco_check_workspace(muloco_ctx* c) {
+  if (!c) return MULOCO_EINVAL;
+  if (c->canary_report.empty()) return MULOCO_OK;
+  const std::string msg = c->canary_report;
+  c->canary_report.clear();
+  return fail(c, MULOCO_ESTATE, "%s", msg.c_str());
 }
 
 MULOCO_API muloco_status muloco_sync_status(muloco_ctx* c) {

@@ -475,6 +475,7 @@ adamw_kernel(const AdamSeg* __restrict__ segs, int n_segs, int64_t n_units, int 
     const int si = find_adam_seg(segs, n_segs, unit);
     const AdamSeg s = segs[si];
     const int64_t base = (unit - s.unit_begin) * ADAM_UNIT;
+    if (!MULOCO_IN_BOUNDS(si >= 0 && si < n_segs && base >= 0 && base < s.n, status)) continue;
     int64_t cnt = s.n - base;
     if (cnt > ADAM_UNIT) cnt = ADAM_UNIT;
     // 16-byte accesses when every stream allows it (bf16 gradients: 8 bytes for the same 4 elements)

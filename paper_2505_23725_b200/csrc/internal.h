@@ -11,6 +11,16 @@ namespace muloco {
 // Device status word bits (OR-ed by kernels, read by muloco_sync_status).
 enum : int { ST_NONFINITE = 1, ST_TIMEOUT = 2, ST_BOUNDS = 4 };
 
+// Debug build (-DMULOCO_DEBUG): kernels check the indices they derive (work-list cursors, matrix
+// slots, tile coordinates, segment and unit indices) before using them; a failed check raises
+// ST_BOUNDS in the status word and the thread skips the access (nothing traps).  In the regular
+// build the checks compile to nothing.
+#ifdef MULOCO_DEBUG
+#define MULOCO_IN_BOUNDS(cond, status) ((cond) ? true : (atomicOr((status), ::muloco::ST_BOUNDS), false))
+#else
+#define MULOCO_IN_BOUNDS(cond, status) (true)
+#endif
+
 // ---------------------------------------------------------------------------
 // Muon path: one entry per (worker, hidden matrix) of a chunk.
 // The Newton-Schulz workspace always holds X as s x l with s <= l; a matrix

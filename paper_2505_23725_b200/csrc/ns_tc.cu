@@ -45,7 +45,7 @@
 // memory: the addend (A for POLY) arrives by TMA, results leave as
 // bulk tensor stores of whole 32 x 64 blocks, so global memory only sees full lines.
 // Every wait is bounded (on a barrier or on a counter): when one runs out the kernel raises
-// ST_TIMEOUT, all roles leave their loops, the CTA frees its tensor memory and returns; the other
+// ST_TIMEOUT (a failed index check of the debug build: ST_BOUNDS), all roles leave their loops, the CTA frees its tensor memory and returns; the other
 // CTAs see the flag in the status word at their next counter wait and leave as well.
 #include <cuda.h>
 #include <stdio.h>
@@ -104,6 +104,7 @@ struct TcMaps {
 struct TcParams {
   const TcBlock* blocks;
   int n_blocks, total_items;
+  int n_mats;                 // matrices of the chunk in this launch
   const int2* tiles_sym;      // (tile row, tile col) in units of 128*CG, tiles on or above the diagonal
   const int2* tiles_full;     // all tiles of the s x l result
   int n_sym, n_full;
@@ -341,25 +342,39 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
 __device__ __forceinline__ Item decode_item(const TcParams& p, int item, int& cur) {
   // items of one worker increase, so the block cursor only moves forward
   const int4* bt = reinterpret_cast<const int4*>(p.blocks);
+  Item q;
+  q.kind = -1;                                  // stays -1 when a debug-build check fails
+  q.ph = q.it = q.m = q.slot = q.N = q.Kd = 0;
+  q.tt = make_int2(0, 0);
+  if (!MULOCO_IN_BOUNDS(cur >= 0 && cur < p.n_blocks, p.status)) return q;
   int4 b0 = __ldg(bt + 2 * cur);
   while (item >= b0.x + b0.y) {
     ++cur;
+    if (!MULOCO_IN_BOUNDS(cur < p.n_blocks, p.status)) return q;
     b0 = __ldg(bt + 2 * cur);
   }
   const int mat0 = __ldg(reinterpret_cast<const int*>(p.blocks) + 8 * cur + 4);
-  Item q;
-  q.kind = b0.z;
-  q.ph = b0.w;
-  q.it = q.ph / 3;
-  const bool sym = q.kind <= GEMM_POLY;
+  const bool sym = b0.z <= GEMM_POLY;
   const int tpm = sym ? p.n_sym : p.n_full;
   const int r = item - b0.x;
   const int ml = r / tpm;
+  q.ph = b0.w;
+  q.it = q.ph / 3;
   q.m = mat0 + ml;
   q.slot = q.m % p.n_slots;
+  if (!MULOCO_IN_BOUNDS(r >= 0 && q.m >= 0 && q.m < p.n_mats && b0.z >= GEMM_GRAM && b0.z <= GEMM_FINAL &&
+                        q.ph >= 0 && q.ph <= p.last_ph, p.status))
+    return q;
   q.tt = (sym ? p.tiles_sym : p.tiles_full)[r - ml * tpm];
   q.N = sym ? p.s : p.l;
-  q.Kd = (q.kind == GEMM_GRAM) ? p.l : p.s;
+  q.Kd = (b0.z == GEMM_GRAM) ? p.l : p.s;
+#ifdef MULOCO_DEBUG
+  {
+    const int T = (p.s > 128) ? 256 : 128;      // tile edge
+    if (!MULOCO_IN_BOUNDS(q.tt.x >= 0 && q.tt.y >= 0 && q.tt.x * T < p.s && q.tt.y * T < q.N, p.status)) return q;
+  }
+#endif
+  q.kind = b0.z;
   return q;
 }
 
@@ -390,7 +405,7 @@ __device__ __forceinline__ bool dep_wait(const TcParams& p, const Item& q, volat
     for (;;) {
       if (ld_acquire(cnt) >= need) break;
       if (*abort_flag) return false;
-      if (ld_acquire(p.status) & ST_TIMEOUT) { *abort_flag = 1; return false; }
+      if (ld_acquire(p.status) & (ST_TIMEOUT | ST_BOUNDS)) { *abort_flag = 1; return false; }
       if (global_timer_ns() - t0 > p.wait_limit_ns) { *abort_flag = 1; return false; }
       __nanosleep(64);
     }
@@ -473,6 +488,7 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       bool withhold = (p.debug_withhold != 0) && (unit == 0);
       for (int item = unit; item < p.total_items && alive; item += n_units) {
         const Item q = decode_item(p, item, cur);
+        if (q.kind < 0) { abort_flag = 2; break; }
         if (!dep_wait<CG>(p, q, &abort_flag)) break;
         const bool sym = q.kind <= GEMM_POLY;
         const bool b_is_x = q.kind >= GEMM_APPLY;             // right operand: X, MN-major
@@ -570,6 +586,7 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       int cur = 0;
       for (int item = unit; item < p.total_items && alive; item += n_units, ++local_tile) {
         const Item q = decode_item(p, item, cur);
+        if (q.kind < 0) { abort_flag = 2; break; }
         const bool sym = q.kind <= GEMM_POLY;
         const bool same = sym && (q.tt.x == q.tt.y);
         const int num_kb = (q.Kd + BK - 1) / BK;
@@ -629,6 +646,7 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     int prev_kind = -1;
     for (int item = unit; item < p.total_items && alive; item += n_units, ++local_tile) {
       const Item q = decode_item(p, item, cur);
+      if (q.kind < 0) { abort_flag = 2; alive = false; break; }
       const int acc = local_tile & 1;
       const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
       const int2 tt = q.tt;
@@ -902,7 +920,7 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     // give copies and MMAs still in flight time to land before memory is released
     const uint64_t t0 = global_timer_ns();
     while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
-    if (threadIdx.x == 0) atomicOr(p.status, ST_TIMEOUT);
+    if (threadIdx.x == 0) atomicOr(p.status, abort_flag == 2 ? ST_BOUNDS : ST_TIMEOUT);
   }
   tc_fence_before();
   if (CG == 2) cluster_sync_all(); else __syncthreads();
@@ -1222,6 +1240,7 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int n_mats, const NsIter
   TcParams p;
   memset(&p, 0, sizeof(p));
   p.blocks = t.dev; p.n_blocks = t.n_blocks; p.total_items = t.total_items;
+  p.n_mats = n_mats;
   p.tiles_sym = pl->tiles_sym; p.tiles_full = pl->tiles_full;
   p.n_sym = pl->n_sym; p.n_full = pl->n_full;
   p.s = (int)pl->s; p.l = (int)pl->l;

@@ -113,11 +113,13 @@ outer_sync_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __
     for (; unit < cta_end; unit += SYNC_WARPS) {
       while (unit >= seg_end) {
         ++seg;
+        if (!MULOCO_IN_BOUNDS(seg < n_segs, status)) return;
         s = segs[seg];
         seg_end = (seg + 1 < n_segs) ? segs[seg + 1].unit_begin : n_units;
         aligned = ((s.cols & 3) == 0) && ((((uintptr_t)s.theta_g | (uintptr_t)s.u) & 15) == 0);
       }
       const int64_t ul = unit - s.unit_begin;
+      if (!MULOCO_IN_BOUNDS(ul >= 0 && ul < s.rows * s.nblk, status)) return;
       const int64_t row = ul / s.nblk;
       const int64_t blk = ul - row * s.nblk;
       const int64_t col0 = blk * block + lane * 4;
@@ -221,10 +223,12 @@ outer_sync2_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* _
     for (; unit < cta_end; unit += SYNC_WARPS) {
       while (unit >= seg_end) {
         ++seg;
+        if (!MULOCO_IN_BOUNDS(seg < n_segs, status)) return;
         s = segs[seg];
         seg_end = (seg + 1 < n_segs) ? segs[seg + 1].unit_begin : n_units;
       }
       const int64_t ul = unit - s.unit_begin;
+      if (!MULOCO_IN_BOUNDS(ul >= 0 && ul < s.rows * s.nblk, status)) return;
       const int64_t row = ul / s.nblk;
       const int64_t blk = ul - row * s.nblk;
       const int64_t col0 = blk * block + lane * 4;
@@ -341,7 +345,7 @@ __device__ __forceinline__ float quant_dequant1(float x, float amax, bool& bad) 
 // worker's delta, or its error-feedback sum) and acc[cols4] (running sum of what the workers sent);
 // every thread only ever touches the entries of its own columns, so the two arrays need no barrier
 // of their own.  Pieces of four columns per thread (16-byte accesses when the row allows it).
-// Rows of up to ROW_PIECES * ROW_THREADS pieces (4096 columns) run software-pipelined: theta stays
+// Without error feedback, rows of up to ROW_PIECES * ROW_THREADS pieces (4096 columns) run software-pipelined: theta stays
 // in registers for the whole row, and the next worker's replica (and accumulator) is already on
 // its way while the current worker's absmax is reduced over the CTA.
 template <int QB, bool EF>
@@ -357,6 +361,7 @@ outer_sync_row1_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* cons
   const int seg = find_seg(segs, n_segs, unit);
   const SyncSeg s = segs[seg];
   const int64_t row = unit - s.unit_begin;
+  if (!MULOCO_IN_BOUNDS(seg >= 0 && seg < n_segs && row >= 0 && row < s.rows, status)) return;
   const int64_t cols = s.cols;
   const int64_t off0 = row * cols;
   float* const* rp = reps + s.rep_index;
@@ -391,8 +396,10 @@ outer_sync_row1_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* cons
   for (int64_t i = threadIdx.x; i < n4; i += ROW_THREADS)
     *reinterpret_cast<float4*>(accb + 4 * i) = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  if (n4 <= (int64_t)ROW_PIECES * ROW_THREADS) {
-    // ---- pipelined: this thread's pieces are i = threadIdx.x + j * ROW_THREADS, j < ROW_PIECES ----
+  if (!EF && n4 <= (int64_t)ROW_PIECES * ROW_THREADS) {
+    // ---- pipelined (without error feedback: with it the accumulators double the registers in
+    // flight and the occupancy lost costs more than the overlap gains: 0.75 against 0.83 of the copy
+    // bandwidth at 4096 columns, K = 16): this thread's pieces are i = threadIdx.x + j * ROW_THREADS, j < ROW_PIECES ----
     float t[ROW_PIECES][4], rv[ROW_PIECES][4], ev[ROW_PIECES][4];
     auto fetch = [&](int k) {
 #pragma unroll
@@ -553,6 +560,7 @@ outer_sync_row_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const
   const int seg = find_seg(segs, n_segs, unit);
   const SyncSeg s = segs[seg];
   const int64_t row = unit - s.unit_begin;
+  if (!MULOCO_IN_BOUNDS(seg >= 0 && seg < n_segs && row >= 0 && row < s.rows, status)) return;
   const int64_t cols = s.cols;
   const int64_t off0 = row * cols;
   float* const* rp = reps + s.rep_index;
