@@ -227,6 +227,10 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--inner", default="muon", choices=["muon", "adamw"],
                     help="adamw: the DiLoCo baseline (AdamW on every tensor) instead of MuLoCo")
+    ap.add_argument("--shard-workers", action="store_true",
+                    help="with --gpus N: spread the workload's K workers over the N ranks (K/N each) and run the outer "
+                         "sync as reduce-scatter + all-gather over NCCL (muloco_shard_*); total work is fixed "
+                         "(strong scaling).  Default: every rank runs its own K-worker problem (weak scaling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workspace-gb", type=float, default=0.0)
@@ -287,6 +291,17 @@ def main():
     torch.cuda.set_device(dev)
 
     seed_init, seed_grad = rank_seeds(w.seed, rank)
+    sharded = bool(args.shard_workers)
+    K_total = w.K
+    if sharded:
+        import dataclasses
+        if w.K % world != 0:
+            raise SystemExit(f"--shard-workers: K={w.K} is not a multiple of {world} ranks")
+        w = dataclasses.replace(w, K=w.K // world)       # this rank's share of the workers
+        seed_init = rank_seeds(w.seed, 0)[0]             # every rank starts from the same global parameters
+        if not distributed:                              # one rank: a communicator of its own
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1"); os.environ.setdefault("MASTER_PORT", "29533")
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(f"cuda:{local_rank}"))
     opt = binding.MuLoCo(w, dev, init_seed=seed_init, alloc_grads=True,
                          workspace_bytes=int(args.workspace_gb * (1 << 30)))
     synth.torch_fill_gradients(opt.grads, w.tensors, w.K, seed_grad, opt.device)
@@ -299,11 +314,16 @@ def main():
             opt.inner_step(-1, None, 1.0)
             t += 1
             for f in opt.fragments_due(t):
-                opt.outer_sync(f)
-                sync_calls[0] += 1
+                if sharded:
+                    wire_bytes[0] += opt.sharded_outer_sync(f, dist)
+                    sync_calls[0] += 3
+                else:
+                    opt.outer_sync(f)
+                    sync_calls[0] += 1
         return t
 
     sync_calls = [0]
+    wire_bytes = [0]
 
     def barrier():
         if distributed:
@@ -317,6 +337,7 @@ def main():
     opt.set_timing(True)
     opt.get_timings()
     sync_calls[0] = 0
+    wire_bytes[0] = 0
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
@@ -335,7 +356,7 @@ def main():
     opt.sync_status()
     ms_total = max_over_ranks(ms_total, dist if distributed else None, dev)
     ms_per_step = ms_total / args.steps
-    units_per_round = w.K * w.n_params * w.H
+    units_per_round = w.K * w.n_params * w.H              # this rank's workers
     value = whole_job_value(world, units_per_round, ms_per_step)
 
     # ---- roofline of the dominant kernel (Newton-Schulz tensor-core GEMMs) ----------------
@@ -387,7 +408,7 @@ def main():
 
     # ---- end to end through the host-buffer entry points ----------------------------------
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not sharded:      # the host-buffer entry points drive the single-GPU sync
         e2e = run_e2e(opt, w, torch, dist if distributed else None, world)
 
     cpu = None
@@ -397,22 +418,31 @@ def main():
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "strong" if sharded else "weak",
                 "vs_baseline": None, "dtype": "bf16" if w.ns_mode == "bf16" else "f32", "data": "synthetic",
                 "config": workload_config(w, args), "clocks": clocks, "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "phases": phase_report}
+        if sharded:
+            line["config"]["parallelism"] = (f"K={K_total} workers spread over {world} ranks ({w.K} each); outer sync = "
+                                             "local delta sums, NCCL reduce-scatter, Nesterov step on the shard, NCCL "
+                                             "all-gather, broadcast into the local replicas")
+            line["sharded_sync"] = {"wire_bytes_per_rank_per_round": wire_bytes[0] / args.steps}
         print(json.dumps(line))
     opt.close()
+    if sharded and not distributed:
+        dist.destroy_process_group()
     if distributed:
         dist.barrier()
         dist.destroy_process_group()
 
 
 def ns_launches_per_inner_step(total_launches, sync_launches, inner_steps, has_adamw):
-    """Newton-Schulz GEMM launches per inner step, from the library's own launch counter: an inner
-    step launches, per workspace chunk, 2 prologue kernels and 15 GEMM kernels, plus one AdamW kernel."""
+    """Newton-Schulz launches per inner step, from the library's own launch counter: an inner step
+    launches, per workspace chunk, 2 staging kernels and 1 kernel that runs all 15 products, plus one
+    AdamW kernel."""
     per_inner = (total_launches - sync_launches) / inner_steps - (1 if has_adamw else 0)
-    return int(round(per_inner / 17.0 * 15.0))
+    return int(round(per_inner / 3.0))
 
 
 def run_ns_only(args):

@@ -182,6 +182,36 @@ MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* ctx, int32_t fragment);
  * may be NULL).  The copies are enqueued on the context's stream. */
 MULOCO_API muloco_status muloco_outer_sync_host(muloco_ctx* ctx, int32_t fragment, void* const* host_theta_g);
 
+/* Worker-sharded outer synchronisation: the K_total = world * K workers of the method are spread
+ * over `world` GPUs (one context per GPU, each holding K of them and its own copy of theta and
+ * u), and Algorithm 1's all-reduce of the outer delta is taken apart into a reduce-scatter and
+ * an all-gather (Section 2, "Collectives for compressed communication"; Appendix, "Assumptions
+ * around the collective used"), which the CALLER runs between the three calls below, on the
+ * context's stream (e.g. NCCL through torch.distributed):
+ *     muloco_shard_delta      stage <- sum over this GPU's workers of (theta - theta_k)
+ *                             (fp32, k ascending; with quant_stages == 2 every worker's delta,
+ *                             or its error-feedback sum, is quantised -> dequantised first)
+ *     reduce-scatter(sum)     stage [stage_floats]  ->  reduced [shard_floats] (shard `rank`)
+ *     muloco_shard_step       Psi = reduced * 1/K_total; the (second) quantisation; Eq. 3 on
+ *                             this GPU's shard of u and theta; theta_shard <- new theta
+ *     all-gather              theta_shard [shard_floats]  ->  theta_all [stage_floats]
+ *     muloco_shard_broadcast  theta and every local replica <- theta_all
+ * Buffers are device float32 arrays in the library's staging layout: unit-major, 128 floats
+ * per unit (a unit is one block of the quantiser, at most 128 elements of one row; unused lanes
+ * hold zeros), padded with zero units so that every GPU's shard has the same number of whole
+ * units; muloco_shard_layout gives the sizes.  u is kept only for the GPU's own shard.  With
+ * world == 1 (no collective) the three calls give what muloco_outer_sync gives, bit for bit;
+ * with more GPUs the sum over GPUs is in the collective's order.  Top-k sparsification and
+ * row-wise quantisation are not available in this form (MULOCO_EINVAL).  Bytes on the wire per
+ * GPU and sync: 2 * 4 * stage_floats * (world - 1) / world. */
+MULOCO_API muloco_status muloco_shard_layout(muloco_ctx* ctx, int32_t fragment, int32_t world, int32_t rank,
+                                             int64_t* stage_floats, int64_t* shard_floats);
+MULOCO_API muloco_status muloco_shard_delta(muloco_ctx* ctx, int32_t fragment, int32_t world, float* stage);
+MULOCO_API muloco_status muloco_shard_step(muloco_ctx* ctx, int32_t fragment, int32_t world, int32_t rank,
+                                           const float* reduced, float* theta_shard);
+MULOCO_API muloco_status muloco_shard_broadcast(muloco_ctx* ctx, int32_t fragment, int32_t world,
+                                                const float* theta_all);
+
 /* Streaming schedule (Section 2, "Partitioned Communication"): fragment j
  * (1-based) is due after inner step t > 0 when t mod H == (j H / J) mod H.
  * Writes the 0-based due fragments to out_frags (host, room for J) and returns

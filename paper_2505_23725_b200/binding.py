@@ -34,6 +34,7 @@ EXPORTS = [
     "muloco_quantize", "muloco_topk_sparsify", "muloco_pseudogradient", "muloco_get_state", "muloco_set_state",
     "muloco_set_timing", "muloco_get_timings", "muloco_sync_status", "muloco_last_error",
     "muloco_newton_schulz_static", "muloco_debug_set", "muloco_check_workspace",
+    "muloco_shard_layout", "muloco_shard_delta", "muloco_shard_step", "muloco_shard_broadcast",
 ]
 
 
@@ -104,6 +105,10 @@ def load_library():
     lib.muloco_last_error.restype = C.c_char_p
     lib.muloco_debug_set.argtypes = [vp, i32, i64]
     lib.muloco_check_workspace.argtypes = [vp]
+    lib.muloco_shard_layout.argtypes = [vp, i32, i32, i32, C.POINTER(i64), C.POINTER(i64)]
+    lib.muloco_shard_delta.argtypes = [vp, i32, i32, vp]
+    lib.muloco_shard_step.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.muloco_shard_broadcast.argtypes = [vp, i32, i32, vp]
     lib.muloco_newton_schulz_static.argtypes = [vp, vp, i32, i64, i64, vp, C.c_char_p, C.c_size_t]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -138,6 +143,48 @@ def newton_schulz_static(X, stream=None, out=None):
     if rc != OK:
         raise MulocoError(rc, err.value.decode())
     return o if X.dim() == 3 else o[0]
+
+
+def shard_wire_bytes(stage_floats: int, world: int) -> int:
+    """Bytes one rank moves per sharded sync: a reduce-scatter and an all-gather of stage_floats
+    float32 values, (world - 1) / world of it each."""
+    return 2 * 4 * stage_floats * (world - 1) // world
+
+
+def _reduce_scatter_sum(dist, out, inp, group):
+    """out <- this rank's shard of the element-wise sum of inp over the ranks."""
+    if dist.get_backend(group) == "nccl":
+        dist.reduce_scatter_tensor(out, inp, op=dist.ReduceOp.SUM, group=group)
+    else:                                   # backends without reduce-scatter (gloo): all-reduce, keep the shard
+        tmp = inp.clone()
+        dist.all_reduce(tmp, op=dist.ReduceOp.SUM, group=group)
+        r = dist.get_rank(group)
+        out.copy_(tmp[r * out.numel():(r + 1) * out.numel()])
+
+
+def sharded_outer_sync(opt, fragment: int, dist, group=None):
+    """Drives the three shard calls of `opt` (a MuLoCo, or any object with shard_layout /
+    shard_delta / shard_step / shard_broadcast and new_buffer) around the two collectives."""
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    stage_floats, shard_floats = opt.shard_layout(fragment, world, rank)
+    if stage_floats == 0:
+        return 0
+    with opt.stream_context():
+        stage = opt.new_buffer(stage_floats)
+        reduced = opt.new_buffer(shard_floats)
+        theta_shard = opt.new_buffer(shard_floats)
+        opt.shard_delta(fragment, world, stage)
+        if world > 1:
+            _reduce_scatter_sum(dist, reduced, stage, group)
+        else:
+            reduced = stage
+        opt.shard_step(fragment, world, rank, reduced, theta_shard)
+        if world > 1:
+            dist.all_gather_into_tensor(stage, theta_shard, group=group)
+        else:
+            stage = theta_shard
+        opt.shard_broadcast(fragment, world, stage)
+    return shard_wire_bytes(stage_floats, world)
 
 
 def make_config(w: _cfg.Workload, workspace_bytes: int = 0, ns_mode: Optional[str] = None, **over) -> Config:
@@ -288,6 +335,12 @@ class MuLoCo:
         self._grad_table_all = _ptr_table([self.grads[k][i].data_ptr() for k in range(self.K)
                                            for i in range(self.n)])
 
+    def new_buffer(self, n: int):
+        return self.torch.empty(n, dtype=self.torch.float32, device=self.device)
+
+    def stream_context(self):
+        return self.torch.cuda.stream(self.stream)
+
     def _check(self, st):
         if st != OK:
             raise MulocoError(st, self.lib.muloco_last_error(self.ctx).decode())
@@ -401,6 +454,31 @@ class MuLoCo:
 
     def sync_status(self):
         self._check(self.lib.muloco_sync_status(self.ctx))
+
+    # -- worker-sharded outer sync: three library calls around the caller's two collectives --------
+    def shard_layout(self, fragment: int, world: int, rank: int):
+        """muloco_shard_layout -> (stage_floats, shard_floats)."""
+        a, b = C.c_int64(0), C.c_int64(0)
+        self._check(self.lib.muloco_shard_layout(self.ctx, fragment, world, rank, C.byref(a), C.byref(b)))
+        return a.value, b.value
+
+    def shard_delta(self, fragment: int, world: int, stage):
+        self._check(self.lib.muloco_shard_delta(self.ctx, fragment, world, stage.data_ptr()))
+
+    def shard_step(self, fragment: int, world: int, rank: int, reduced, theta_shard):
+        self._check(self.lib.muloco_shard_step(self.ctx, fragment, world, rank, reduced.data_ptr(),
+                                               theta_shard.data_ptr()))
+
+    def shard_broadcast(self, fragment: int, world: int, theta_all):
+        self._check(self.lib.muloco_shard_broadcast(self.ctx, fragment, world, theta_all.data_ptr()))
+
+    def sharded_outer_sync(self, fragment: int, dist, group=None):
+        """The outer synchronisation with the workers spread over the ranks of `group`
+        (torch.distributed): local delta sums -> reduce-scatter -> Nesterov step on the shard ->
+        all-gather -> broadcast into the local replicas.  The collectives run on this context's
+        stream.  Returns the bytes this rank sent and received over the wire (the ring
+        algorithm's 2 * 4 * stage_floats * (world - 1) / world)."""
+        return sharded_outer_sync(self, fragment, dist, group)
 
     def check_workspace(self):
         """muloco_check_workspace: raises MulocoError(ESTATE) if a workspace canary was overwritten."""

@@ -927,6 +927,87 @@ MULOCO_API muloco_status muloco_outer_sync_host(muloco_ctx* c, int32_t fragment,
   return MULOCO_OK;
 }
 
+// ---- worker-sharded outer synchronisation ------------------------------------------------
+namespace {
+muloco_status shard_check(muloco_ctx* c, int32_t fragment, int32_t world, int32_t rank, FragTable** ft) {
+  if (!c) return MULOCO_EINVAL;
+  const muloco_config& f = c->cfg;
+  if (fragment < -1 || fragment >= f.J) return fail(c, MULOCO_EINVAL, "fragment %d outside -1..%d", fragment, f.J - 1);
+  if (world < 1 || rank < 0 || rank >= world) return fail(c, MULOCO_EINVAL, "bad world/rank (%d, %d)", world, rank);
+  if (f.topk_fraction > 0.f) return fail(c, MULOCO_EINVAL, "the sharded sync does not do top-k sparsification");
+  if (f.quant != MULOCO_Q_NONE && f.quant_block == 0)
+    return fail(c, MULOCO_EINVAL, "the sharded sync does not do row-wise quantisation");
+  *ft = &c->frags[fragment < 0 ? f.J : fragment];
+  return MULOCO_OK;
+}
+int64_t shard_units(int64_t n_units, int32_t world) { return (n_units + world - 1) / world; }
+}  // namespace
+
+MULOCO_API muloco_status muloco_shard_layout(muloco_ctx* c, int32_t fragment, int32_t world, int32_t rank,
+                                             int64_t* stage_floats, int64_t* shard_floats) {
+  FragTable* ft = nullptr;
+  const muloco_status s = shard_check(c, fragment, world, rank, &ft);
+  if (s != MULOCO_OK) return s;
+  const int64_t us = shard_units(ft->n_units, world);
+  if (stage_floats) *stage_floats = us * world * 128;
+  if (shard_floats) *shard_floats = us * 128;
+  return MULOCO_OK;
+}
+
+MULOCO_API muloco_status muloco_shard_delta(muloco_ctx* c, int32_t fragment, int32_t world, float* stage) {
+  FragTable* ft = nullptr;
+  const muloco_status s = shard_check(c, fragment, world, 0, &ft);
+  if (s != MULOCO_OK) return s;
+  if (ft->n_segs == 0) return MULOCO_OK;
+  if (!stage) return fail(c, MULOCO_EINVAL, "stage is NULL");
+  const muloco_config& f = c->cfg;
+  PhaseTimer t(c, MULOCO_PH_SYNC);
+  const int64_t us = shard_units(ft->n_units, world);
+  const int64_t pad = us * world - ft->n_units;      // units that only make the shards equal: zeros
+  if (pad > 0) CK(cudaMemsetAsync(stage + ft->n_units * 128, 0, (size_t)pad * 128 * sizeof(float), c->st));
+  const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
+  launch_shard_delta(c->st, ft->d_segs, ft->n_segs, c->d_replicas, f.K, ft->n_units, blk, f.quant,
+                     f.quant_stages == 2 ? 2 : 1, c->d_ef, f.ef_beta, stage, c->d_status);
+  c->launches += 1;
+  CK(cudaGetLastError());
+  return MULOCO_OK;
+}
+
+MULOCO_API muloco_status muloco_shard_step(muloco_ctx* c, int32_t fragment, int32_t world, int32_t rank,
+                                           const float* reduced, float* theta_shard) {
+  FragTable* ft = nullptr;
+  const muloco_status s = shard_check(c, fragment, world, rank, &ft);
+  if (s != MULOCO_OK) return s;
+  if (ft->n_segs == 0) return MULOCO_OK;
+  if (!reduced || !theta_shard) return fail(c, MULOCO_EINVAL, "reduced or theta_shard is NULL");
+  const muloco_config& f = c->cfg;
+  PhaseTimer t(c, MULOCO_PH_SYNC);
+  const int64_t us = shard_units(ft->n_units, world);
+  const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
+  const float inv_k_total = 1.0f / (float)((int64_t)f.K * world);
+  launch_shard_step(c->st, ft->d_segs, ft->n_segs, ft->n_units, us * rank, us, blk, f.quant, f.outer_lr,
+                    f.outer_momentum, inv_k_total, reduced, theta_shard, c->d_status);
+  c->launches += 1;
+  CK(cudaGetLastError());
+  return MULOCO_OK;
+}
+
+MULOCO_API muloco_status muloco_shard_broadcast(muloco_ctx* c, int32_t fragment, int32_t world, const float* theta_all) {
+  FragTable* ft = nullptr;
+  const muloco_status s = shard_check(c, fragment, world, 0, &ft);
+  if (s != MULOCO_OK) return s;
+  const muloco_config& f = c->cfg;
+  if (fragment < 0) for (auto& n : c->frag_syncs) n += 1; else c->frag_syncs[fragment] += 1;
+  if (ft->n_segs == 0) return MULOCO_OK;
+  if (!theta_all) return fail(c, MULOCO_EINVAL, "theta_all is NULL");
+  PhaseTimer t(c, MULOCO_PH_SYNC);
+  const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
+  launch_shard_broadcast(c->st, ft->d_segs, ft->n_segs, c->d_replicas, f.K, ft->n_units, blk, theta_all, c->d_status);
+  c->launches += 1;
+  CK(cudaGetLastError());
+  return MULOCO_OK;
+}
+
 MULOCO_API int32_t muloco_fragments_due(const muloco_ctx* c, int64_t step, int32_t* out_frags) {
   if (!c || !out_frags) return -1;
   if (step <= 0) return 0;

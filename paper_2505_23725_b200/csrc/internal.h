@@ -126,6 +126,16 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
 cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
                                    int K, int64_t n_rows, int64_t max_cols, int quant_bits, float outer_lr,
                                    float mu, int* status, int stages, float* const* ef, float ef_beta);
+// Worker-sharded outer synchronisation (outer_sync.cu): the three passes around the caller's
+// reduce-scatter and all-gather.  Staging buffers are unit-major, 128 floats per unit.
+void launch_shard_delta(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,
+                        int64_t n_units, int block, int quant_bits, int stages, float* const* ef, float ef_beta,
+                        float* stage, int* status);
+void launch_shard_step(cudaStream_t st, const SyncSeg* segs, int n_segs, int64_t n_units, int64_t unit_begin,
+                       int64_t unit_count, int block, int quant_bits, float outer_lr, float mu, float inv_k_total,
+                       const float* reduced, float* theta_out, int* status);
+void launch_shard_broadcast(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,
+                            int64_t n_units, int block, const float* theta_all, int* status);
 // Top-k sparsification of the workers' deltas (topk.cu).  Scratch: one histogram of
 // topk_hist_words_per_problem() words (zero between calls), one prefix word (the threshold key
 // after a call) and one counter per (tensor, worker), indexed like the replica table.

@@ -706,6 +706,186 @@ void launch_sync_q(cudaStream_t st, dim3 grid, const SyncSeg* segs, int n_segs, 
 #undef MULOCO_SYNC_CASE
 }
 
+// ---------------------------------------------------------------------------
+// Worker-sharded outer synchronisation: the workers are partitioned over G GPUs and the all-reduce
+// of the outer delta (Algorithm 1) is taken apart into a reduce-scatter and an all-gather (Section 2,
+// "Collectives for compressed communication"; Appendix, "Assumptions around the collective used").
+// Three passes on each GPU, the two collectives between them are the caller's:
+//   delta     : S = sum over this GPU's workers of (theta - theta_k) (fp32, k ascending; with two
+//               quantisation stages every worker's delta, or error-feedback sum, is quantised ->
+//               dequantised first)                                 -> staging buffer, then reduce-scatter
+//   step      : on this GPU's shard: Psi = (sum over all GPUs) * 1/K_total, the (second)
+//               quantisation, u and theta updated in place      -> new theta of the shard, then all-gather
+//   broadcast : theta and every local replica <- gathered theta.
+// The staging buffers are unit-major with a fixed stride of 128 floats per unit (a unit is a
+// block of the quantiser, at most 128 elements of one row; lanes beyond a short block hold zeros), so
+// a shard is a range of whole units and every GPU gets the same count.
+// ---------------------------------------------------------------------------
+struct UnitPos {
+  int64_t off;      // element offset of this lane's four values inside the tensor
+  int nvalid;
+  bool vec;
+};
+
+__device__ __forceinline__ UnitPos unit_pos(const SyncSeg& s, int64_t unit, int block, int lane) {
+  const int64_t ul = unit - s.unit_begin;
+  const int64_t row = ul / s.nblk;
+  const int64_t blk = ul - row * s.nblk;
+  const int64_t col0 = blk * block + lane * 4;
+  int64_t blk_end = (blk + 1) * block;
+  if (blk_end > s.cols) blk_end = s.cols;
+  int nvalid = (int)(blk_end - col0);
+  nvalid = nvalid < 0 ? 0 : (nvalid > 4 ? 4 : nvalid);
+  UnitPos p;
+  p.off = row * s.cols + col0;
+  p.nvalid = nvalid;
+  p.vec = (nvalid == 4) && ((s.cols & 3) == 0) && ((((uintptr_t)s.theta_g | (uintptr_t)s.u) & 15) == 0);
+  return p;
+}
+
+template <int QB, bool TWO, bool EF>
+__global__ void __launch_bounds__(SYNC_THREADS)
+shard_delta_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps,
+                   float* const* __restrict__ efs, int K, int64_t n_units, int64_t units_per_cta, int block,
+                   float ef_beta, float* __restrict__ stage, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t cta_begin = (int64_t)blockIdx.x * units_per_cta;
+  int64_t cta_end = cta_begin + units_per_cta;
+  if (cta_end > n_units) cta_end = n_units;
+  bool bad = false;
+  for (int64_t unit = cta_begin + warp; unit < cta_end; unit += SYNC_WARPS) {
+    const int seg = find_seg(segs, n_segs, unit);
+    if (!MULOCO_IN_BOUNDS(seg >= 0 && seg < n_segs, status)) return;
+    const SyncSeg s = segs[seg];
+    if (!MULOCO_IN_BOUNDS(unit - s.unit_begin < s.rows * s.nblk, status)) return;
+    UnitPos u = unit_pos(s, unit, block, lane);
+    float* const* rp = reps + s.rep_index;
+    float* const* ep = EF ? efs + s.rep_index : nullptr;
+    for (int k = 0; k < K; ++k) {
+      u.vec = u.vec && ((((uintptr_t)rp[k]) & 15) == 0);
+      if (EF) u.vec = u.vec && ((((uintptr_t)ep[k]) & 15) == 0);
+    }
+    float tg[4] = {0.f, 0.f, 0.f, 0.f}, acc[4] = {0.f, 0.f, 0.f, 0.f};
+    if (u.nvalid > 0) load4(s.theta_g + u.off, u.vec, u.nvalid, tg);
+    for (int k0 = 0; k0 < K; k0 += 4) {
+      float r[4][4], e[EF ? 4 : 1][4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { r[j][q] = 0.f; e[EF ? j : 0][q] = 0.f; }
+        if (k0 + j < K && u.nvalid > 0) {
+          load4(rp[k0 + j] + u.off, u.vec, u.nvalid, r[j]);
+          if (EF) load4(ep[k0 + j] + u.off, u.vec, u.nvalid, e[EF ? j : 0]);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (k0 + j < K) {              // uniform over the warp: the block reduction needs every lane
+          float x[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float d = __fsub_rn(tg[q], r[j][q]);
+            x[q] = EF ? __fadd_rn(__fmul_rn(ef_beta, e[EF ? j : 0][q]), d) : d;
+          }
+          float sent[4] = {x[0], x[1], x[2], x[3]};
+          if (TWO) {
+            int qq[4]; float sc;
+            quant_dequant4<(QB == 0 ? 8 : QB)>(sent, u.nvalid, qq, sc, bad);
+            if (EF && u.nvalid > 0) {
+              float en[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) en[q] = __fsub_rn(x[q], sent[q]);
+              store4(ep[k0 + j] + u.off, u.vec, u.nvalid, en);
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], sent[q]);
+        }
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (q >= u.nvalid) acc[q] = 0.f;
+    __stcs(reinterpret_cast<float4*>(stage + unit * 128 + lane * 4), make_float4(acc[0], acc[1], acc[2], acc[3]));
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
+}
+
+template <int QB>
+__global__ void __launch_bounds__(SYNC_THREADS)
+shard_step_kernel(const SyncSeg* __restrict__ segs, int n_segs, int64_t n_units, int64_t unit_begin,
+                  int64_t unit_count, int block, float eta, float mu, float inv_k_total,
+                  const float* __restrict__ reduced, float* __restrict__ theta_out, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t j = (int64_t)blockIdx.x * SYNC_WARPS + (threadIdx.x >> 5);
+  if (j >= unit_count) return;
+  const int64_t unit = unit_begin + j;
+  bool bad = false;
+  float tn[4] = {0.f, 0.f, 0.f, 0.f};
+  if (unit < n_units) {                   // beyond: padding units that make the shards equal
+    const int seg = find_seg(segs, n_segs, unit);
+    if (!MULOCO_IN_BOUNDS(seg >= 0 && seg < n_segs, status)) return;
+    const SyncSeg s = segs[seg];
+    if (!MULOCO_IN_BOUNDS(unit - s.unit_begin < s.rows * s.nblk, status)) return;
+    const UnitPos u = unit_pos(s, unit, block, lane);
+    const float4 rv = __ldcs(reinterpret_cast<const float4*>(reduced + j * 128 + lane * 4));
+    float psi[4] = {__fmul_rn(rv.x, inv_k_total), __fmul_rn(rv.y, inv_k_total), __fmul_rn(rv.z, inv_k_total),
+                    __fmul_rn(rv.w, inv_k_total)};
+    if (QB != 0) {
+      int q[4]; float sc;
+      quant_dequant4<(QB == 0 ? 8 : QB)>(psi, u.nvalid, q, sc, bad);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e < u.nvalid && !(fabsf(psi[e]) <= FLT_MAX)) bad = true;
+    }
+    if (u.nvalid > 0) {
+      float tg[4], uu[4], un[4];
+      load4(s.theta_g + u.off, u.vec, u.nvalid, tg);
+      load4(s.u + u.off, u.vec, u.nvalid, uu);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float ep = eta * psi[e];
+        un[e] = fmaf(mu, uu[e], ep);
+        tn[e] = tg[e] - fmaf(mu, un[e], ep);
+      }
+      store4(s.u + u.off, u.vec, u.nvalid, un);
+      store4(s.theta_g + u.off, u.vec, u.nvalid, tn);
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e >= u.nvalid) tn[e] = 0.f;
+    }
+  }
+  __stcs(reinterpret_cast<float4*>(theta_out + j * 128 + lane * 4), make_float4(tn[0], tn[1], tn[2], tn[3]));
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
+}
+
+__global__ void __launch_bounds__(SYNC_THREADS)
+shard_broadcast_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps, int K,
+                       int64_t n_units, int64_t units_per_cta, int block, const float* __restrict__ theta_all,
+                       int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t cta_begin = (int64_t)blockIdx.x * units_per_cta;
+  int64_t cta_end = cta_begin + units_per_cta;
+  if (cta_end > n_units) cta_end = n_units;
+  for (int64_t unit = cta_begin + warp; unit < cta_end; unit += SYNC_WARPS) {
+    const int seg = find_seg(segs, n_segs, unit);
+    if (!MULOCO_IN_BOUNDS(seg >= 0 && seg < n_segs, status)) return;
+    const SyncSeg s = segs[seg];
+    if (!MULOCO_IN_BOUNDS(unit - s.unit_begin < s.rows * s.nblk, status)) return;
+    UnitPos u = unit_pos(s, unit, block, lane);
+    if (u.nvalid == 0) continue;
+    float* const* rp = reps + s.rep_index;
+    for (int k = 0; k < K; ++k) u.vec = u.vec && ((((uintptr_t)rp[k]) & 15) == 0);
+    const float4 v = __ldcs(reinterpret_cast<const float4*>(theta_all + unit * 128 + lane * 4));
+    const float tn[4] = {v.x, v.y, v.z, v.w};
+    store4(s.theta_g + u.off, u.vec, u.nvalid, tn);
+    for (int k = 0; k < K; ++k) store4(rp[k] + u.off, u.vec, u.nvalid, tn);
+  }
+}
+
 }  // namespace
 
 void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
@@ -741,6 +921,47 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
     launch_sync_q<2>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
   else
     launch_sync_q<0>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+}
+
+void launch_shard_delta(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,
+                        int64_t n_units, int block, int quant_bits, int stages, float* const* ef, float ef_beta,
+                        float* stage, int* status) {
+  if (n_units <= 0) return;
+  const int64_t upc = (int64_t)SYNC_WARPS * SYNC_UNITS_PER_WARP;
+  dim3 grid((unsigned)((n_units + upc - 1) / upc));
+  const bool two = (stages == 2 && quant_bits != 0);
+#define MULOCO_SD(QB, TWO, EF)                                                                             \
+  shard_delta_kernel<QB, TWO, EF><<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, replicas, ef, K, n_units, upc, \
+                                                                block, ef_beta, stage, status)
+  if (!two) MULOCO_SD(0, false, false);
+  else if (quant_bits == 8) { if (ef) MULOCO_SD(8, true, true); else MULOCO_SD(8, true, false); }
+  else if (quant_bits == 4) { if (ef) MULOCO_SD(4, true, true); else MULOCO_SD(4, true, false); }
+  else { if (ef) MULOCO_SD(2, true, true); else MULOCO_SD(2, true, false); }
+#undef MULOCO_SD
+}
+
+void launch_shard_step(cudaStream_t st, const SyncSeg* segs, int n_segs, int64_t n_units, int64_t unit_begin,
+                       int64_t unit_count, int block, int quant_bits, float outer_lr, float mu, float inv_k_total,
+                       const float* reduced, float* theta_out, int* status) {
+  if (unit_count <= 0) return;
+  dim3 grid((unsigned)((unit_count + SYNC_WARPS - 1) / SYNC_WARPS));
+#define MULOCO_SS(QB)                                                                                       \
+  shard_step_kernel<QB><<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, n_units, unit_begin, unit_count, block, \
+                                                        outer_lr, mu, inv_k_total, reduced, theta_out, status)
+  if (quant_bits == 8) MULOCO_SS(8);
+  else if (quant_bits == 4) MULOCO_SS(4);
+  else if (quant_bits == 2) MULOCO_SS(2);
+  else MULOCO_SS(0);
+#undef MULOCO_SS
+}
+
+void launch_shard_broadcast(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,
+                            int64_t n_units, int block, const float* theta_all, int* status) {
+  if (n_units <= 0) return;
+  const int64_t upc = (int64_t)SYNC_WARPS * SYNC_UNITS_PER_WARP;
+  dim3 grid((unsigned)((n_units + upc - 1) / upc));
+  shard_broadcast_kernel<<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, replicas, K, n_units, upc, block, theta_all,
+                                                        status);
 }
 
 cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
