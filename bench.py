@@ -31,12 +31,20 @@ if ROOT not in sys.path:
 METRIC = "optimizer-step params/sec (inner Muon + outer sync) at K workers"
 UNIT = "param-updates/s"
 
-# DRAM traffic of the Newton-Schulz GEMM launches per hidden-matrix parameter, worker and inner
-# step, from the ncu capture summarised in profiles/ns_tc_kernel_muon-only_K16_L2_d1024_F2816.md
-# (19.91 GB over the 30 launches of a 2-layer, K=16 inner step with 25,690,112 parameters per
-# replica).  It grows in proportion to the number of matrices, so it is scaled by the parameter
-# count; it holds for the d=1024, F=2816 shape mix only.
-NS_TRAFFIC_BYTES_PER_PARAM = {(1024, 2816): 19.909e9 / (25690112 * 16)}
+# Measured constants of the Newton-Schulz kernel (one launch = all 15 products of a chunk), quoted
+# beside the live timings.  Source: one `ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,
+# sm__pipe_tensor_cycles_active...` capture per shape mix of `bench.py --muon-only K 2 D F` (two
+# layers, the configuration's K; both launches of an inner step).  Key: (d_model, ff).
+#   bytes: DRAM bytes read + written per hidden-matrix parameter, worker and inner step.  Traffic
+#          grows in proportion to the number of matrices, so a full launch is this figure times the
+#          parameters it covers.
+#   tensor_pct: sm__pipe_tensor_cycles_active, % of peak, of the two launches (square group, wide group).
+NS_KERNEL_COUNTERS = {
+    (768, 2048): {"bytes": 4.18708e9 / (14155776 * 8), "tensor_pct": (45.5, 53.7)},
+    (1024, 2816): {"bytes": 15.93625e9 / (25690112 * 16), "tensor_pct": (56.7, 57.4)},
+    (2048, 5632): {"bytes": 35.31191e9 / (102760448 * 8), "tensor_pct": (67.7, 68.6)},
+    (3072, 8192): {"bytes": 45.64105e9 / (226492416 * 4), "tensor_pct": (67.1, 67.5)},
+}
 
 
 def load_peaks():
@@ -374,13 +382,22 @@ def main():
             if tn.name.endswith(".w1"):
                 shape_key = (tn.rows, tn.cols)
                 break
-        per_param = NS_TRAFFIC_BYTES_PER_PARAM.get(shape_key)
-        traffic = (per_param * w.n_muon_params * w.K / ns_launches_per_inner) if per_param else None
-        roofline = {"bound": "tensor", "kernel": "ns_tc_kernel (Gram / polynomial / apply GEMMs of Newton-Schulz)",
+        counters = NS_KERNEL_COUNTERS.get(shape_key)
+        traffic = (counters["bytes"] * w.n_muon_params * w.K / ns_launches_per_inner) if counters else None
+        executed = ns_tflops * w.ns_flops_executed() / w.ns_flops_credited()
+        roofline = {"bound": "tensor", "kernel": "ns_tc_kernel (all Gram / polynomial / apply products of Newton-Schulz)",
                     "achieved": ns_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": ns_tflops / peak_tf,
                     "peak_source": f"{peaks['source']} sustained bf16 matmul (kernel timed inside a long step)",
+                    "frac_of_burst_peak": ns_tflops / peaks["bf16_tflops"],
+                    "frac_of_nominal_2250": ns_tflops / 2250.0,
+                    "executed_tflops": executed, "executed_frac": executed / peak_tf,
                     "launches_per_inner_step": ns_launches_per_inner,
-                    "traffic": traffic, "traffic_unit": "bytes per launch (average over the launches of an inner step)",
+                    "traffic": traffic,
+                    "traffic_unit": "bytes per launch (average over the launches of an inner step)" if counters else
+                                    "null: no counter capture exists for this shape mix",
+                    "tensor_pipe_pct_ncu": list(counters["tensor_pct"]) if counters else None,
+                    "tensor_pipe_source": "sm__pipe_tensor_cycles_active of the 2-layer case of this shape mix, "
+                                          "launch alone (square group, wide group)",
                     "flops_convention": "credited 5*(4 s^2 l + 2 s^3) per matrix; symmetric products run upper-triangle tiles only",
                     "ms_per_inner_step": ns_ms_per_inner}
     else:
@@ -389,7 +406,8 @@ def main():
         gbs = adam_bytes / (phases["adamw"] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "adamw_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} copy bandwidth",
-                    "traffic": adam_bytes / inner_steps, "traffic_unit": "bytes per launch (= algorithmic, see profiles/)"}
+                    "traffic": adam_bytes / inner_steps,
+                    "traffic_unit": "bytes per launch (ncu: DRAM traffic of this kernel equals its algorithmic bytes)"}
     n_sync_rounds = args.steps
     sync_gbs = w.sync_bytes() * n_sync_rounds / (phases["sync"] * 1e-3) / 1e9 if phases["sync"] > 0 else None
     adam_gbs = adam_bytes / (phases["adamw"] * 1e-3) / 1e9 if phases["adamw"] > 0 else None
@@ -578,7 +596,8 @@ def run_elementwise_only(args):
 def run_e2e(opt, w, torch, dist, world):
     """The same round through muloco_inner_step_host / muloco_outer_sync_host: every inner
     step copies that step's gradients from pinned host memory, every sync reads the new
-    global parameters back to the host.  One warm-up inner step, one timed round."""
+    global parameters back to the host.  One warm-up inner step, two timed rounds (both reported;
+    the value is their mean)."""
     import psutil
     elt = 2 if w.grad_dtype == "bf16" else 4
     set_bytes = opt.flat_numel * elt
@@ -596,26 +615,30 @@ def run_e2e(opt, w, torch, dist, world):
     out = [out_flat[o:o + t.numel].view(t.rows, t.cols) for o, t in zip(opt.offsets, w.tensors)]
     opt.inner_step_host(-1, host, 1.0)
     torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    e0.record(opt.stream)
-    t = 0
-    d2h = 0
-    for _ in range(w.H):
-        opt.inner_step_host(-1, host, 1.0)
-        t += 1
-        for f in opt.fragments_due(t):
-            opt.outer_sync_host(f, out)
-            d2h += sum(tt.numel for tt in w.tensors if tt.fragment == f) * 4
-    e1.record(opt.stream)
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    ms = max_over_ranks(ms, dist, opt.device)
+    rounds = 2
+    per_round, d2h, t = [], 0, 0
+    for _ in range(rounds):
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(opt.stream)
+        d2h = 0
+        for _ in range(w.H):
+            opt.inner_step_host(-1, host, 1.0)
+            t += 1
+            for f in opt.fragments_due(t):
+                opt.outer_sync_host(f, out)
+                d2h += sum(tt.numel for tt in w.tensors if tt.fragment == f) * 4
+        e1.record(opt.stream)
+        torch.cuda.synchronize()
+        per_round.append(max_over_ranks(e0.elapsed_time(e1), dist, opt.device))
     opt.sync_status()
+    ms = sum(per_round) / len(per_round)
     h2d = w.n_params * elt * w.K * w.H
     return {"value": whole_job_value(world, w.K * w.n_params * w.H, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "rounds_timed": 1, "host_grad_sets": n_sets}
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "rounds_timed": rounds, "ms_per_round": per_round,
+            "host_grad_sets": n_sets}
 
 
 if __name__ == "__main__":

@@ -20,6 +20,13 @@
  *     return value at once.  Conditions found on the device (non-finite
  *     pseudogradient, a bounded wait that ran out) are written to a device
  *     status word and reported by muloco_sync_status.  Nothing aborts or traps.
+ *   - Accuracy, against the definitions evaluated in exact arithmetic on the same float32 state:
+ *     the element-wise steps (momentum, AdamW, outer step) are within
+ *     |err| <= 1e-6 * |x| + 1e-6 * rms(tensor) per element -- the second term is an absolute
+ *     floor, wider than "1e-6 relative" for entries far below the tensor's root mean square,
+ *     where one float32 rounding of a sum of larger terms already exceeds 1e-6 of the entry;
+ *     quantiser codes, scales and dequantised values are exact; Newton-Schulz: see
+ *     muloco_newton_schulz.
  *   - Calls on one context are not thread-safe.
  *   - There is no CPU fallback: without a CUDA device every compute call
  *     returns MULOCO_ECUDA.
@@ -281,10 +288,11 @@ MULOCO_API muloco_status muloco_newton_schulz_static(const float* X, float* O, i
 MULOCO_API muloco_status muloco_quantize(muloco_ctx* ctx, const float* psi, int64_t rows, int64_t cols,
                               int32_t bits, int8_t* codes, float* scales, float* dequant);
 
-/* The top-k sparsifier on its own (Section 2, "Compressed Communication"): x and out are
+/* Test hook: the top-k sparsifier on its own (Section 2, "Compressed Communication"): x and out are
  * DEVICE arrays of n float32 (they may be the same array); out = x where |x| is at least the
  * kk-th largest magnitude, kk = max(1, floor(fraction * n)), else 0.  fraction in (0, 1].
- * Allocates and frees a few KB of device scratch; waits for the stream before returning. */
+ * Not for a hot path: it allocates and frees a few KB of device scratch and waits for the
+ * stream before returning (the synchronisation's own scratch is allocated once, at create). */
 MULOCO_API muloco_status muloco_topk_sparsify(muloco_ctx* ctx, const float* x, int64_t n, float fraction,
                                    float* out);
 
@@ -304,7 +312,8 @@ enum {
   MULOCO_PH_NS = 1,       /* Newton-Schulz GEMMs, including the fused final update    */
   MULOCO_PH_ADAMW = 2,
   MULOCO_PH_SYNC = 3,
-  MULOCO_PH_COPY = 4,     /* host<->device copies of the *_host calls                 */
+  MULOCO_PH_COPY = 4,     /* host<->device copies of the *_host calls (sum over the two
+                             copy streams, which run side by side)                    */
   MULOCO_N_PHASES = 5
 };
 MULOCO_API muloco_status muloco_set_timing(muloco_ctx* ctx, int32_t enabled);

@@ -110,7 +110,7 @@ WsLayout make_layout(int64_t s, int64_t ldx, int64_t lds, int chunk, int n_part,
   }
   w.partials = place("partials", (size_t)chunk * n_part * sizeof(float));
   w.scales = place("scales", (size_t)chunk * sizeof(float2));
-  w.counters = place("counters", (size_t)chunk * 3 * ns_steps * sizeof(int));
+  w.counters = place("counters", ((size_t)chunk * 3 * ns_steps + 16) * sizeof(int));   // tile counters + ticket
   w.total = align_up(off + WS_GUARD, 1024);
   return w;
 }
@@ -713,7 +713,8 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
     for (int i = 0; i < n; ++i)
       if (!grads[(size_t)(k - k0) * n + i]) return fail(c, MULOCO_EINVAL, "gradient of tensor %d (worker %d) is NULL", i, k);
   if (n == 0) return MULOCO_OK;
-  for (int k = k0; k < k1; ++k) c->worker_step[k] += 1;
+  // the step counters advance only once the whole step has been enqueued (a call that fails on the
+  // way leaves them, and with them AdamW's bias correction and the state blob, where they were)
   const int g_is_bf16 = (f.grad_dtype == MULOCO_BF16);
 
   char* host = nullptr;
@@ -747,7 +748,7 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
   size_t na = 0;
   int64_t units = 0;
   for (int k = k0; k < k1; ++k) {
-    const double t_step = (double)c->worker_step[k];
+    const double t_step = (double)(c->worker_step[k] + 1);
     const double bc1 = f.adam_bias_correction ? 1.0 - pow((double)f.adam_beta1, t_step) : 1.0;
     const double bc2 = f.adam_bias_correction ? 1.0 - pow((double)f.adam_beta2, t_step) : 1.0;
     for (int i : c->adam_ids) {
@@ -806,6 +807,7 @@ MULOCO_API muloco_status muloco_inner_step(muloco_ctx* c, int32_t worker, const 
     }
   }
   CK(cudaGetLastError());
+  for (int k = k0; k < k1; ++k) c->worker_step[k] += 1;
   return MULOCO_OK;
 }
 
@@ -859,7 +861,9 @@ MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* c, int32_t worker, c
       CK(cudaStreamWaitEvent(c->copy_st2, c->ev_consumed[sec], 0));
     }
     {
+      // both copy streams are timed; the reported copy phase is the sum of their busy spans
       PhaseTimer t(c, MULOCO_PH_COPY, c->copy_st);
+      PhaseTimer t2(c, MULOCO_PH_COPY, c->copy_st2);
       int which = 0;
       for (int k = k0; k < k1; ++k)
         for (int i : ids) {

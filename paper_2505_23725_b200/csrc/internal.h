@@ -75,7 +75,7 @@ struct TcGroupPlan;   // opaque per-shape-group plan (tensor maps, tile lists, w
 int tc_group_size(int64_t s, int chunk);
 // bytes of the ring (X', X'', A, B for n_slots matrices, bf16)
 size_t tc_ring_bytes(int64_t s, int64_t ldx, int64_t lds, int n_slots);
-// counters: chunk * 3 * ns_steps ints (zeroed by every launch)
+// counters: chunk * 3 * ns_steps + 1 ints (tile counters and the ticket counter; zeroed by every launch)
 TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, int64_t ldx, void* ring, int64_t lds,
                             int group, int* counters, int ns_steps, char* err, size_t errlen);
 void tc_plan_destroy(TcGroupPlan*);

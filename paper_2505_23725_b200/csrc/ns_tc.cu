@@ -17,14 +17,15 @@
 // intermediates (X', A, B') live in a small ring of 2 D slots that the next group but one reuses;
 // only the first Gram and the first apply read the staged input from its chunk-sized buffer.
 //
-// Work items go to the tile workers round-robin (item i to worker i mod W), every worker takes its
-// items in increasing order, and all workers are resident at once.  An item only depends on items
-// before it in the list: a product of matrix m needs all tiles of m's previous product (and the
-// first product of m needs the ring slot's previous user to be finished).  Finished tiles are
-// counted per (matrix, product) in global memory: every epilogue warp adds one (release) once its
-// part of the tile is in memory; the TMA producer (and, for the polynomial's addend, the epilogue)
-// waits (acquire) until the count of the product it reads is complete.  The item with the smallest
-// index that is not finished always has its inputs ready, so the list drains.
+// The tile workers (CTA pairs) take the items in list order from a ticket counter in global memory, and
+// all workers are resident at once.  An item only depends on items before it in the list: a product of
+// matrix m needs all tiles of m's previous product (and the first product of m needs the ring slot's
+// previous user to be finished).  Finished tiles are counted per (matrix, product) in global memory:
+// every epilogue warp adds one (release) once its part of the tile is in memory; a worker's
+// dispatcher thread claims the next item, waits (acquire) until the count of the product it reads is
+// complete and only then hands the item to the worker's other roles.  The unfinished item with the
+// smallest index always has its inputs ready, so the list drains; a worker that has to wait for an
+// input delays only itself, the others go on claiming items.
 // Operand forms: GRAM/POLY multiply a row-major matrix by its own transpose
 // (both operands K-major); APPLY needs X with the contraction index as the slow
 // axis, i.e. an MN-major B operand, so no transposed copy of X is ever made.
@@ -38,9 +39,12 @@
 //            rows.  No load is multicast: each CTA fetches its own slabs.
 //   CG = 1 : one CTA, 128 x 128 tiles (matrices with at most 128 rows).
 //
-// CTA = 6 warps: warp 0 issues TMA loads, warp 1 allocates tensor memory and
+// CTA = 7 warps: warp 0 issues TMA loads, warp 1 allocates tensor memory and
 // (rank 0) issues the MMAs, warps 2-5 run the epilogue (one 32-lane quarter of
-// the accumulator each).  Two accumulators alternate so the epilogue of one
+// the accumulator each), warp 6 is the dispatcher: one thread (of the rank-0 CTA) that claims and
+// decodes the worker's items, waits for their inputs and publishes them in a shared-memory ring of
+// both CTAs, one item ahead of the producer, so that no other role ever waits on global memory
+// between two tiles.  Two accumulators alternate so the epilogue of one
 // tile overlaps the main loop of the next.  The epilogue goes through shared
 // memory: the addend (A for POLY) arrives by TMA, results leave as
 // bulk tensor stores of whole 32 x 64 blocks, so global memory only sees full lines.
@@ -65,7 +69,7 @@ namespace {
 constexpr int BM = 128;          // rows per CTA (one CTA's share of UMMA M)
 constexpr int BK = 64;           // k slab per stage (64 bf16 = one 128-byte swizzle row)
 constexpr int UMMA_K = 16;
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 224;      // 7 warps: producer, MMA issuer, 4 epilogue warps, scout
 constexpr int TC_STAGES = 5;
 // Five pipeline stages beside four staging blocks per epilogue warp (GRAM, APPLY: results; POLY:
 // addend + results; FINAL: the parameter ring).
@@ -116,11 +120,12 @@ struct TcParams {
   int sink_mode;
   int x_wide, s_wide;         // the _MN maps of X / of A and B are the 4-D form (both 64-column atoms of a slab in one copy)
   int n_slots;
+  int* ticket;                // next unclaimed item (zeroed by every launch)
   int* counters;              // [chunk][cw]: epilogue warps that have finished product ph of matrix m
   int cw;
   int* status;
   unsigned long long wait_limit_ns;
-  int debug_withhold;         // test hook: worker 0 never issues the first operand copy of its first item
+  int debug_withhold;         // test hook: the first operand copy of the list's first item is never issued
 };
 
 // One work item, as every role decodes it.
@@ -422,6 +427,63 @@ __device__ __forceinline__ void signal_done(const TcParams& p, const Item& q) {
   asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
 }
 
+// ---- the item ring --------------------------------------------------------------------------
+// The dispatcher (one thread of the worker: warp 6, lane 0 of the rank-0 CTA) claims the worker's next
+// item from a ticket counter in global memory, decodes it, waits for its inputs and then publishes
+// it, packed into 64 bits, in a ring in shared memory of every CTA of the worker (for the peer CTA
+// through distributed shared memory).  The other roles read their n-th item from slot n % RING.
+//   bits 63..52 tag = (n + 1) mod 4096 | 51..44 ph | 43..22 m | 21..14 tile row | 13..0 tile column
+// ph = RING_STOP marks the end of the work.  A slot is rewritten RING items later; the dispatcher stays
+// at most one item ahead of the producer, the producer at most TC_STAGES tiles ahead of the MMA
+// issuer (a tile is at least one k slab) and the MMA issuer at most two tiles ahead of the epilogue
+// (two accumulators), so no reader is ever RING items behind.
+constexpr int RING = 16;
+constexpr int RING_STOP = 255;
+
+__device__ __forceinline__ uint64_t ring_pack(int n, int ph, int m, int tx, int ty) {
+  return ((uint64_t)((n + 1) & 0xFFF) << 52) | ((uint64_t)(ph & 0xFF) << 44) | ((uint64_t)(m & 0x3FFFFF) << 22) |
+         ((uint64_t)(tx & 0xFF) << 14) | (uint64_t)(ty & 0x3FFF);
+}
+__device__ __forceinline__ void ring_store(uint32_t cluster_addr, uint64_t v) {
+  asm volatile("st.release.cluster.shared::cluster.b64 [%0], %1;" ::"r"(cluster_addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint64_t ring_load(uint32_t addr) {
+  uint64_t v;
+  asm volatile("ld.acquire.cluster.shared::cta.b64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+  return v;
+}
+// The worker's n-th item, once the dispatcher has published it.  Called by one thread; kind = -1 when
+// the CTA is aborting, kind = -2 at the end of the work.
+__device__ __forceinline__ Item ring_read(const TcParams& p, uint32_t ring0, int n, volatile int* abort_flag,
+                                          uint64_t limit_ns) {
+  const uint32_t addr = ring0 + (uint32_t)(n % RING) * 8u;
+  const uint64_t tag = (uint64_t)((n + 1) & 0xFFF);
+  uint64_t v = ring_load(addr);
+  Item q;
+  q.kind = -1; q.ph = q.it = q.m = q.slot = q.N = q.Kd = 0; q.tt = make_int2(0, 0);
+  if ((v >> 52) != tag) {
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+      v = ring_load(addr);
+      if ((v >> 52) == tag) break;
+      if (*abort_flag) return q;
+      if (global_timer_ns() - t0 > limit_ns) { *abort_flag = 1; return q; }
+    }
+  }
+  q.ph = (int)((v >> 44) & 0xFF);
+  if (q.ph == RING_STOP) { q.kind = -2; return q; }
+  q.it = q.ph / 3;
+  q.m = (int)((v >> 22) & 0x3FFFFF);
+  q.slot = q.m % p.n_slots;
+  q.tt = make_int2((int)((v >> 14) & 0xFF), (int)(v & 0x3FFF));
+  const int r3 = q.ph - 3 * q.it;
+  q.kind = (r3 == 0) ? GEMM_GRAM : (r3 == 1) ? GEMM_POLY : (q.ph == p.last_ph ? GEMM_FINAL : GEMM_APPLY);
+  const bool sym = r3 < 2;
+  q.N = sym ? p.s : p.l;
+  q.Kd = (r3 == 0) ? p.l : p.s;
+  return q;
+}
+
 // ------------------------------- the kernel --------------------------------
 template <int CG>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -440,17 +502,19 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   __shared__ __align__(8) uint64_t bar_w[4][4];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile int abort_flag;
+  __shared__ __align__(8) uint64_t item_ring[RING];      // written by the dispatcher (of rank 0)
+  __shared__ int prod_started;                           // rank 0: tiles the producer has begun
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;
-  const int unit = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // tile worker index
-  const int n_units = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint64_t limit = p.wait_limit_ns;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
+    prod_started = 0;
+    for (int i = 0; i < RING; ++i) item_ring[i] = 0;
 #pragma unroll 1
     for (int i = 0; i < N_MAPS; ++i) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[i]) : "memory");
     for (int s = 0; s < STAGES; ++s) {
@@ -484,12 +548,15 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       const uint32_t full0_bar = (CG == 2) ? map_to_rank(full0, 0) : full0;
       uint32_t stage = 0, phase = 0;
       bool alive = true;
-      int cur = 0;
-      bool withhold = (p.debug_withhold != 0) && (unit == 0);
-      for (int item = unit; item < p.total_items && alive; item += n_units) {
-        const Item q = decode_item(p, item, cur);
-        if (q.kind < 0) { abort_flag = 2; break; }
-        if (!dep_wait<CG>(p, q, &abort_flag)) break;
+      const uint32_t ring0 = smem_u32(&item_ring[0]);
+      const uint32_t started_addr = smem_u32(&prod_started);
+      for (int n_local = 0; alive; ++n_local) {
+        const Item q = ring_read(p, ring0, n_local, &abort_flag, limit);
+        if (q.kind < 0) break;                               // end of the work, or aborting
+        // the dispatcher may now claim the item after this one
+        if (rank == 0) asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(started_addr), "r"(n_local + 1) : "memory");
+        // what the other CTAs wrote through the async proxy is read through the async proxy next
+        asm volatile("fence.proxy.async;" ::: "memory");
         const bool sym = q.kind <= GEMM_POLY;
         const bool b_is_x = q.kind >= GEMM_APPLY;             // right operand: X, MN-major
         const bool same = sym && (q.tt.x == q.tt.y);          // diagonal tile: right slab == left slab
@@ -521,6 +588,8 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         const int ka_mn = (q.kind != GEMM_GRAM) ? (TM / BK) * q.tt.x : 0;
         const int kb_mn = (q.kind == GEMM_POLY) ? (TM / BK) * q.tt.y : 0;
         const int num_kb = (q.Kd + BK - 1) / BK;
+        // test hook: the first k slab of the very first item of the list
+        bool withhold = (p.debug_withhold != 0) && q.ph == 0 && q.m == 0 && q.tt.x == 0 && q.tt.y == 0;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty0 + stage * 8u, phase ^ 1u, &abort_flag, limit)) { alive = false; break; }
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
@@ -583,10 +652,10 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       uint32_t stage = 0, phase = 0;
       int local_tile = 0;
       bool alive = true;
-      int cur = 0;
-      for (int item = unit; item < p.total_items && alive; item += n_units, ++local_tile) {
-        const Item q = decode_item(p, item, cur);
-        if (q.kind < 0) { abort_flag = 2; break; }
+      const uint32_t ring0 = smem_u32(&item_ring[0]);
+      for (; alive; ++local_tile) {
+        const Item q = ring_read(p, ring0, local_tile, &abort_flag, limit);
+        if (q.kind < 0) break;
         const bool sym = q.kind <= GEMM_POLY;
         const bool same = sym && (q.tt.x == q.tt.y);
         const int num_kb = (q.Kd + BK - 1) / BK;
@@ -624,6 +693,44 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       }
     }
     __syncwarp();
+  } else if (warp == 6) {
+    // ------------------------------- dispatcher -------------------------------
+    if (rank == 0 && lane == 0) {
+      const uint32_t ring0 = smem_u32(&item_ring[0]);
+      const uint32_t ring0_peer = (CG == 2) ? map_to_rank(ring0, 1) : 0u;
+      const uint32_t started_addr = smem_u32(&prod_started);
+      auto publish = [&](int n, uint64_t v) {
+        ring_store(ring0 + (uint32_t)(n % RING) * 8u, v);
+        if (CG == 2) ring_store(ring0_peer + (uint32_t)(n % RING) * 8u, v);
+      };
+      int cur = 0;
+      for (int n = 0;; ++n) {
+        // stay one item ahead of the producer: item n is claimed once the producer has begun item n - 2
+        if (n >= 2) {
+          int st;
+          asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(st) : "r"(started_addr) : "memory");
+          if (st < n - 1) {
+            const uint64_t t0 = global_timer_ns();
+            bool ok = true;
+            for (;;) {
+              asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(st) : "r"(started_addr) : "memory");
+              if (st >= n - 1) break;
+              if (abort_flag) { ok = false; break; }
+              if (global_timer_ns() - t0 > limit) { abort_flag = 1; ok = false; break; }
+              __nanosleep(32);
+            }
+            if (!ok) break;
+          }
+        }
+        const int item = atomicAdd(p.ticket, 1);
+        if (item >= p.total_items) { publish(n, ring_pack(n, RING_STOP, 0, 0, 0)); break; }
+        const Item q = decode_item(p, item, cur);
+        if (q.kind < 0) { abort_flag = 2; break; }
+        if (!dep_wait<CG>(p, q, &abort_flag)) break;
+        publish(n, ring_pack(n, q.ph, q.m, q.tt.x, q.tt.y));
+      }
+    }
+    __syncwarp();
   } else {
     // -------------------------------- epilogue --------------------------------
     const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter+32)
@@ -642,11 +749,22 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     uint32_t cin_issued = 0, cin_used = 0, st_count = 0, t_count = 0;
     int local_tile = 0;
     bool alive = true;
-    int cur = 0;
     int prev_kind = -1;
-    for (int item = unit; item < p.total_items && alive; item += n_units, ++local_tile) {
-      const Item q = decode_item(p, item, cur);
-      if (q.kind < 0) { abort_flag = 2; alive = false; break; }
+    const uint32_t ring0 = smem_u32(&item_ring[0]);
+    for (; alive; ++local_tile) {
+      // lane 0 reads the ring, the packed item goes to the other lanes by shuffle
+      Item q;
+      {
+        Item q0;
+        q0.kind = 0; q0.ph = q0.it = q0.m = q0.slot = q0.N = q0.Kd = 0; q0.tt = make_int2(0, 0);
+        if (lane == 0) q0 = ring_read(p, ring0, local_tile, &abort_flag, limit);
+        q.kind = __shfl_sync(0xffffffffu, q0.kind, 0); q.ph = __shfl_sync(0xffffffffu, q0.ph, 0);
+        q.it = __shfl_sync(0xffffffffu, q0.it, 0);     q.m = __shfl_sync(0xffffffffu, q0.m, 0);
+        q.slot = __shfl_sync(0xffffffffu, q0.slot, 0); q.N = __shfl_sync(0xffffffffu, q0.N, 0);
+        q.Kd = __shfl_sync(0xffffffffu, q0.Kd, 0);
+        q.tt.x = __shfl_sync(0xffffffffu, q0.tt.x, 0); q.tt.y = __shfl_sync(0xffffffffu, q0.tt.y, 0);
+      }
+      if (q.kind < 0) { alive = false; break; }
       const int acc = local_tile & 1;
       const uint32_t acc_phase = (uint32_t)(local_tile >> 1) & 1u;
       const int2 tt = q.tt;
@@ -691,11 +809,9 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         ++cin_issued;
       };
       if (has_cin && todo) {
-        // the addend is the Gram matrix of this iteration: wait until all of its tiles are in memory
-        int ok = 1;
-        if (lane == 0) ok = dep_wait<CG>(p, q, &abort_flag) ? 1 : 0;
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) { alive = false; break; }
+        // the addend is the Gram matrix of this iteration: the item was only published once all of its
+        // tiles were in memory
+        if (lane == 0) asm volatile("fence.proxy.async;" ::: "memory");
         issue_cin(__ffs(todo) - 1);
       }
       // fused parameter update: the old parameters come in as 32 x 32 blocks, two steps ahead
@@ -1235,7 +1351,8 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int n_mats, const NsIter
   BlockTable t;
   cudaError_t e = get_table(pl, n_mats, &t);
   if (e != cudaSuccess) return e;
-  e = cudaMemsetAsync(pl->counters, 0, (size_t)n_mats * pl->cw * sizeof(int), st);
+  // tile counters and, behind them, the ticket counter
+  e = cudaMemsetAsync(pl->counters, 0, ((size_t)n_mats * pl->cw + 1) * sizeof(int), st);
   if (e != cudaSuccess) return e;
   TcParams p;
   memset(&p, 0, sizeof(p));
@@ -1250,6 +1367,7 @@ cudaError_t tc_launch(cudaStream_t st, TcGroupPlan* pl, int n_mats, const NsIter
   p.x_wide = pl->wide_x; p.s_wide = pl->wide_s;
   p.n_slots = pl->n_slots;
   p.counters = pl->counters; p.cw = pl->cw;
+  p.ticket = pl->counters + (size_t)n_mats * pl->cw;
   p.status = args.status;
   p.wait_limit_ns = args.wait_limit_ns ? args.wait_limit_ns : 2000000000ull;
   p.debug_withhold = args.debug_withhold;
