@@ -34,7 +34,7 @@ struct WsRegion { const char* name; size_t off, bytes; };
 
 struct WsLayout {   // byte offsets inside the workspace for one shape group
   // fp32 engine: x0, x1, a, b are chunk-sized.  bf16 engine: x0 is the chunk-sized staged input and
-  // `ring` holds the intermediates of 2 * group matrices; `counters` counts finished tiles.
+  // `ring` holds the intermediates of tc_ring_slots(group) matrices; `counters` counts finished tiles.
   // Every region lies between guard zones of at least 1 KB; the 64 bytes right before and right
   // after a region are its canaries (see muloco_check_workspace).
   size_t x0 = 0, x1 = 0, a = 0, b = 0, ring = 0, partials = 0, scales = 0, counters = 0, total = 0;
@@ -48,7 +48,7 @@ struct Group {
   int n_part = 0;
   int elt = 2;
   int mode = MULOCO_NS_BF16;   // engine that serves this group (see engine_for)
-  int ring_group = 1;          // bf16 engine: matrices per group of the work list (ring = 2 * ring_group slots)
+  int ring_group = 1;          // bf16 engine: matrices per group of the work list (the ring has tc_ring_slots(ring_group) slots)
   WsLayout ws;
   TcGroupPlan* plan = nullptr;
 };
@@ -101,7 +101,7 @@ WsLayout make_layout(int64_t s, int64_t ldx, int64_t lds, int chunk, int n_part,
   const size_t xb = (size_t)chunk * s * ldx * elt;
   w.x0 = place("X0", xb);
   if (elt == 2) {
-    w.ring = place("ring", tc_ring_bytes(s, ldx, lds, 2 * ring_group));
+    w.ring = place("ring", tc_ring_bytes(s, ldx, lds, tc_ring_slots(ring_group)));
   } else {
     const size_t sb = (size_t)chunk * s * lds * elt;
     w.x1 = place("X1", xb);
@@ -134,7 +134,7 @@ void size_group(int64_t s, int64_t l, int64_t ldx, int64_t lds, int64_t count, s
   size_t fixed = 0;
   if (elt == 2) {
     rg = tc_group_size(s, (int)std::min<int64_t>(count, 1 << 30));
-    fixed = tc_ring_bytes(s, ldx, lds, 2 * rg);
+    fixed = tc_ring_bytes(s, ldx, lds, tc_ring_slots(rg));
   }
   const size_t per_slot = make_layout(s, ldx, lds, 1, np, elt, 0, ns_steps).total;
   const size_t avail = budget > fixed + per_slot ? budget - fixed : per_slot;

@@ -69,11 +69,12 @@ void launch_ns_fp32(cudaStream_t st, int kind, int n_mats, int64_t s, int64_t l,
 
 // bf16 tensor-core engine (tcgen05 / TMEM / TMA); see ns_tc.cu.  One launch runs all products of
 // all iterations for the matrices of a chunk; the staged input X0 is chunk-sized, the
-// intermediates live in a ring of 2 * group slots.
+// intermediates live in a ring of tc_ring_slots(group) slots.
 struct TcGroupPlan;   // opaque per-shape-group plan (tensor maps, tile lists, work lists)
 // matrices per group of the work list for min-dimension s (never more than `chunk`)
 int tc_group_size(int64_t s, int chunk);
-// bytes of the ring (X', X'', A, B for n_slots matrices, bf16)
+// ring slots for groups of `group` matrices; bytes of the ring (X', X'', A, B for n_slots matrices, bf16)
+int tc_ring_slots(int group);
 size_t tc_ring_bytes(int64_t s, int64_t ldx, int64_t lds, int n_slots);
 // counters: chunk * 3 * ns_steps + 1 ints (tile counters and the ticket counter; zeroed by every launch)
 TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, int64_t ldx, void* ring, int64_t lds,

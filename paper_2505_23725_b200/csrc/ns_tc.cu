@@ -1177,7 +1177,7 @@ struct TcGroupPlan {
   int64_t s, l, ldx, lds;
   int chunk;
   int cg;                       // CTAs per tile worker (1 or 2)
-  int group, n_slots;           // matrices per group of the work list, ring slots (2 * group)
+  int group, n_slots;           // matrices per group of the work list, ring slots (tc_ring_slots(group))
   int ns_steps, cw;
   TcMaps maps;
   bool wide_x = false, wide_s = false;
@@ -1199,17 +1199,18 @@ int tc_num_sms() {
   return n;
 }
 
-// Matrices per group of the work list.  Between the tiles of one product of a matrix and the tiles
-// of its next product lie the same product's tiles of the group's other matrices; with about two
-// rounds of the tile workers in between, a worker (and its copies, which run a tile ahead) rarely
-// finds its inputs unfinished.  More matrices per group would only push the intermediates out of L2.
+// Matrices per group of the work list: about one round of the tile workers per block of a symmetric
+// product (at least two matrices).  Measured on the four benchmark shape mixes (Newton-Schulz ms per
+// inner step against the group size): smaller groups leave a product's tiles still running when the
+// matrix's next product comes up, larger ones push the intermediates out of L2.
 int tc_group_size(int64_t s, int chunk) {
   const int cg = (s > 128) ? 2 : 1;
   const int64_t T = 128 * cg;
   const int64_t tm = (s + T - 1) / T;
   const int64_t n_sym = tm * (tm + 1) / 2;
   const int units = tc_num_sms() / cg;
-  int64_t g = (2 * units + n_sym - 1) / n_sym;
+  int64_t g = (units + n_sym - 1) / n_sym;
+  if (g < 2) g = 2;
   if (const char* e = getenv("MULOCO_NS_GROUP")) {     // tuning studies
     const int v = atoi(e);
     if (v > 0) g = v;
@@ -1218,6 +1219,10 @@ int tc_group_size(int64_t s, int chunk) {
   if (g > chunk) g = chunk;
   return (int)g;
 }
+
+// Three groups are in flight at a time (see get_table) and a fourth set of slots belongs to the group
+// that finished last, so that a new group never waits for its slots.
+int tc_ring_slots(int group) { return 4 * group; }
 
 size_t tc_ring_bytes(int64_t s, int64_t ldx, int64_t lds, int n_slots) {
   const size_t xb = ((size_t)n_slots * s * ldx * 2 + 1023) / 1024 * 1024;
@@ -1229,7 +1234,7 @@ TcGroupPlan* tc_plan_create(int64_t s, int64_t l, int chunk, void* X0, int64_t l
                             int group, int* counters, int ns_steps, char* err, size_t errlen) {
   TcGroupPlan* pl = new TcGroupPlan();
   pl->s = s; pl->l = l; pl->ldx = ldx; pl->lds = lds; pl->chunk = chunk;
-  pl->group = group; pl->n_slots = 2 * group;
+  pl->group = group; pl->n_slots = tc_ring_slots(group);
   pl->ns_steps = ns_steps; pl->cw = 3 * ns_steps;
   pl->counters = counters;
   pl->n_sms = tc_num_sms();
@@ -1308,17 +1313,30 @@ void tc_plan_destroy(TcGroupPlan* pl) {
 
 namespace {
 
-// The work list for the first n_mats matrices of the chunk: groups of `group` matrices, each group
-// product by product (Gram, polynomial, apply of iteration 0, 1, ...), each product matrix by matrix.
+// The work list for the first n_mats matrices of the chunk.  The matrices are taken in groups of
+// `group`; a group runs its products one after the other (Gram, polynomial, apply of iteration 0, 1,
+// ...), one block per product, matrix by matrix inside a block.  Three groups are in flight, a third
+// of the products apart: in step t of the list, group g is at product t - (n_ph / 3) g.  With five
+// iterations (15 products) the three groups of a step are at a Gram, a polynomial and an apply,
+// so between a product of a matrix and its next product always lie two blocks of other groups,
+// one of them of a long kind, and the matrices in flight stay few (3 * group).
 cudaError_t get_table(TcGroupPlan* pl, int n_mats, BlockTable* out) {
   auto it = pl->tables.find(n_mats);
   if (it != pl->tables.end()) { *out = it->second; return cudaSuccess; }
   std::vector<TcBlock> blocks;
   int64_t item = 0;
-  const int last_ph = pl->cw - 1;
-  for (int g0 = 0; g0 < n_mats; g0 += pl->group) {
-    const int n = (n_mats - g0 < pl->group) ? (n_mats - g0) : pl->group;
-    for (int ph = 0; ph <= last_ph; ++ph) {
+  const int n_ph = pl->cw;
+  const int last_ph = n_ph - 1;
+  const int n_groups = (n_mats + pl->group - 1) / pl->group;
+  const int lag = (n_ph + 2) / 3;                            // steps between the starts of two groups
+  const int n_steps = (n_groups - 1) * lag + n_ph;
+  for (int t = 0; t < n_steps; ++t) {
+    for (int g = 0; g < n_groups; ++g) {
+      const int ph = t - g * lag;
+      if (ph < 0) break;
+      if (ph > last_ph) continue;
+      const int g0 = g * pl->group;
+      const int n = (n_mats - g0 < pl->group) ? (n_mats - g0) : pl->group;
       TcBlock b;
       memset(&b, 0, sizeof b);
       b.kind = (ph % 3 == 0) ? GEMM_GRAM : (ph % 3 == 1) ? GEMM_POLY : (ph == last_ph ? GEMM_FINAL : GEMM_APPLY);
