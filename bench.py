@@ -40,10 +40,10 @@ UNIT = "param-updates/s"
 #          parameters it covers.
 #   tensor_pct: sm__pipe_tensor_cycles_active, % of peak, of the two launches (square group, wide group).
 NS_KERNEL_COUNTERS = {
-    (768, 2048): {"bytes": 4.18708e9 / (14155776 * 8), "tensor_pct": (45.5, 53.7)},
-    (1024, 2816): {"bytes": 15.93625e9 / (25690112 * 16), "tensor_pct": (56.7, 57.4)},
-    (2048, 5632): {"bytes": 35.31191e9 / (102760448 * 8), "tensor_pct": (67.7, 68.6)},
-    (3072, 8192): {"bytes": 45.64105e9 / (226492416 * 4), "tensor_pct": (67.1, 67.5)},
+    (768, 2048): {"bytes": 4.36606e9 / (14155776 * 8), "tensor_pct": (47.3, 56.8)},
+    (1024, 2816): {"bytes": 17.98357e9 / (25690112 * 16), "tensor_pct": (64.8, 69.5)},
+    (2048, 5632): {"bytes": 38.66371e9 / (102760448 * 8), "tensor_pct": (76.4, 78.7)},
+    (3072, 8192): {"bytes": 48.34281e9 / (226492416 * 4), "tensor_pct": (79.6, 80.3)},
 }
 
 

@@ -705,16 +705,18 @@ ns_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       };
       int cur = 0;
       for (int n = 0;; ++n) {
-        // stay one item ahead of the producer: item n is claimed once the producer has begun item n - 2
-        if (n >= 2) {
+        // stay one item ahead of the producer: item n is claimed once the producer has begun item n - 1
+        // (claiming further ahead was measured slower: a claimed item that waits behind its worker's
+        // current tile holds up the items that depend on it)
+        if (n >= 1) {
           int st;
           asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(st) : "r"(started_addr) : "memory");
-          if (st < n - 1) {
+          if (st < n) {
             const uint64_t t0 = global_timer_ns();
             bool ok = true;
             for (;;) {
               asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(st) : "r"(started_addr) : "memory");
-              if (st >= n - 1) break;
+              if (st >= n) break;
               if (abort_flag) { ok = false; break; }
               if (global_timer_ns() - t0 > limit) { abort_flag = 1; ok = false; break; }
               __nanosleep(32);
