@@ -232,7 +232,8 @@ MULOCO_API int32_t muloco_fragments_due(const muloco_ctx* ctx, int64_t step, int
  * ns_mode MULOCO_NS_BF16 runs the tensor-core engine (bf16 operands, fp32
  * accumulation), MULOCO_NS_FP32 the fp32 engine.  X and O must not overlap.
  * Accuracy against the iteration in exact arithmetic (relative Frobenius error):
- * 1e-4 for the fp32 engine, 2e-2 for the bf16 engine.  The bf16 engine holds its
+ * 1e-4 for the fp32 engine, 2e-2 for the bf16 engine with up to the paper's five steps (more
+ * steps amplify the roundings of the earlier ones: 2.4e-2 was seen with seven).  The bf16 engine holds its
  * bound only from min(rows, cols) = 64 on; matrices with a smaller min-dimension
  * (also inside muloco_inner_step) are always served by the fp32 engine, whatever
  * mode is asked, and meet the fp32 bound. */

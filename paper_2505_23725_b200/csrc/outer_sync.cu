@@ -207,7 +207,8 @@ outer_sync2_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* _
                    float eta, float mu, float inv_k, float ef_beta, int* __restrict__ status) {
   // workers per batch (their loads are in flight together).  Measured at 400M parameters, int4:
   // without error feedback 2 beats 4, 8, 16 (K=16: 5.64 / 5.56 / 4.91 / 5.42 TB/s; K=5: 5.27 / 4.81 / 4.11 /
-  // 3.88), with error feedback 4 beats 2, 8, 16 (6.42 / 5.84 / 6.08 / 4.15 TB/s).
+  // 3.88), with error feedback 4 beats 2, 8, 16 (6.42 / 5.84 / 6.08 / 4.15 TB/s).  Fetching the next batch
+  // before the current one is reduced (double-buffered registers) was slower in both (4.94 and 5.60 TB/s).
   constexpr int WB = EF ? 4 : 2;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;

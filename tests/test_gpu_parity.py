@@ -600,6 +600,49 @@ def test_nonfinite_gradient_of_an_adamw_tensor_is_reported(grad_dtype):
 
 
 # ---------------------------------------------------------------------------
+# the work list of the tensor-core kernel away from its defaults
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("steps", [1, 2, 3, 7])
+def test_newton_schulz_with_other_iteration_counts(steps):
+    import torch
+    w = configs.Workload("ns-only", K=1, H=1, J=1, tensors=[], muon_lr=0.02, muon_beta=0.95, muon_wd=0.0,
+                         outer_lr=1.0, outer_momentum=0.0)
+    ctx = gpu_for(w, [], ns_steps=steps)
+    rng = np.random.default_rng(60 + steps)
+    for batch, m, n in [(3, 256, 384), (2, 200, 96), (5, 128, 128)]:
+        X = np.stack([synth.lowrank_plus_noise(rng, m, n) for _ in range(batch)])
+        # the bf16 bound is stated for the paper's five steps; every further step amplifies the roundings
+        # of the earlier ones in the directions that are still converging
+        for mode, tol in (("fp32", 1e-4), ("bf16", 2e-2 if steps <= 5 else 4e-2)):
+            out = _np(ctx.newton_schulz(torch.from_numpy(X).cuda(), ns_mode=mode))
+            ctx.sync_status()
+            for b in range(batch):
+                ref = O.newton_schulz(X[b], steps=steps)
+                assert relfro(out[b], ref) < tol, f"{steps} steps {mode} {m}x{n}: {relfro(out[b], ref):.3e}"
+    ctx.close()
+
+
+@pytest.mark.parametrize("group", [1, 2, 3])
+def test_tiny_groups_and_tiny_chunks_reuse_ring_slots_many_times(monkeypatch, group):
+    """Groups of 1-3 matrices (ring of 4-12 slots) and a workspace of a few MB: 45 matrices go through
+    several chunks and every ring slot is reused many times, with the dependency of a group's first
+    product on the slot's previous user in play."""
+    import torch
+    monkeypatch.setenv("MULOCO_NS_GROUP", str(group))
+    w = configs.Workload("ns-only", K=1, H=1, J=1, tensors=[], muon_lr=0.02, muon_beta=0.95, muon_wd=0.0,
+                         outer_lr=1.0, outer_momentum=0.0)
+    ctx = gpu_for(w, [], workspace_bytes=10 << 20)
+    rng = np.random.default_rng(90 + group)
+    for batch, m, n in [(45, 256, 384), (33, 384, 130), (20, 128, 640)]:
+        X = np.stack([synth.lowrank_plus_noise(rng, m, n) * (10.0 ** rng.uniform(-2, 2)) for _ in range(batch)])
+        out = _np(ctx.newton_schulz(torch.from_numpy(X).cuda(), ns_mode="bf16"))
+        ctx.sync_status()
+        for b in range(batch):
+            assert relfro(out[b], O.newton_schulz(X[b])) < 2e-2, f"group {group} {m}x{n} matrix {b}"
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------
 # failure path of the tensor-core kernel: a wait that runs out (nothing faults, nothing hangs)
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("batch,m,n", [(1, 256, 256), (1, 128, 128), (40, 512, 768), (3, 64, 200)])
