@@ -27,6 +27,11 @@
  *     where one float32 rounding of a sum of larger terms already exceeds 1e-6 of the entry;
  *     quantiser codes, scales and dequantised values are exact; Newton-Schulz: see
  *     muloco_newton_schulz.
+ *   - The tensor-core Newton-Schulz kernel is one persistent launch whose thread blocks hand
+ *     tiles to one another; it needs all of them resident at once, i.e. the GPU to itself while it
+ *     runs (kernels of the same stream are fine: they run before or after).  If another context
+ *     or stream holds SMs for long, its waits run out and the call ends with MULOCO_ETIMEOUT
+ *     instead of hanging.
  *   - Calls on one context are not thread-safe.
  *   - There is no CPU fallback: without a CUDA device every compute call
  *     returns MULOCO_ECUDA.
