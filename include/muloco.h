@@ -184,6 +184,9 @@ MULOCO_API muloco_status muloco_inner_step_host(muloco_ctx* ctx, int32_t worker,
  *               ascending, then * 1/K) and quantised -> dequantised again
  *     u <- mu u + eta_out Psi;   theta_g <- theta_g - mu u - eta_out Psi
  *     theta_k <- theta_g for every worker.
+ * With K == 1, eta_out == 1, mu == 0 and no compression (plain data parallelism, Section 5's DP
+ * baselines) the step is the identity on the worker: theta_g <- theta_1 bit for bit (H plain
+ * inner steps, exactly), u <- theta_g - theta_1, one pass of 16 bytes per parameter.
  * Inner optimizer state is kept.  Syncing a fragment that is not due is allowed;
  * the schedule is the caller's (see muloco_fragments_due). */
 MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* ctx, int32_t fragment);

@@ -897,6 +897,13 @@ MULOCO_API muloco_status muloco_outer_sync(muloco_ctx* c, int32_t fragment) {
     CK(cudaGetLastError());
     return MULOCO_OK;
   }
+  if (f.K == 1 && f.quant == MULOCO_Q_NONE && f.outer_lr == 1.0f && f.outer_momentum == 0.0f) {
+    // plain data parallelism (Section 5's DP baselines): the outer step is the identity on theta_1
+    launch_dp_sync(c->st, ft.d_segs, ft.n_segs, c->d_replicas, ft.n_units, c->d_status);
+    c->launches += 1;
+    CK(cudaGetLastError());
+    return MULOCO_OK;
+  }
   const int blk = (f.quant == MULOCO_Q_NONE) ? 128 : f.quant_block;
   if (f.quant != MULOCO_Q_NONE && blk == 0) {
     cudaError_t e = launch_outer_sync_rows(c->st, ft.d_segs, ft.n_segs, c->d_replicas, f.K, ft.n_units, ft.max_cols,

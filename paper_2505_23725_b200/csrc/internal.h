@@ -127,6 +127,9 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
 cudaError_t launch_outer_sync_rows(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
                                    int K, int64_t n_rows, int64_t max_cols, int quant_bits, float outer_lr,
                                    float mu, int* status, int stages, float* const* ef, float ef_beta);
+// K = 1, eta_out = 1, mu = 0, no compression: theta <- theta_1 (exactly), u <- theta - theta_1.
+void launch_dp_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int64_t n_units,
+                    int* status);
 // Worker-sharded outer synchronisation (outer_sync.cu): the three passes around the caller's
 // reduce-scatter and all-gather.  Staging buffers are unit-major, 128 floats per unit.
 void launch_shard_delta(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,

@@ -887,6 +887,42 @@ shard_broadcast_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* cons
   }
 }
 
+// Plain data parallelism as a special case (Section 5, the DP baselines): one worker, eta_out = 1,
+// mu = 0, no compression.  Eq. 3 then gives theta <- theta - (theta - theta_1) = theta_1 in exact
+// arithmetic, so the worker's parameters are copied (exactly: H plain inner steps), u <- theta - theta_1,
+// and the replica is left as it is: 16 instead of 24 bytes per parameter.
+__global__ void __launch_bounds__(SYNC_THREADS)
+dp_sync_kernel(const SyncSeg* __restrict__ segs, int n_segs, float* const* __restrict__ reps, int64_t n_units,
+               int64_t units_per_cta, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t cta_begin = (int64_t)blockIdx.x * units_per_cta;
+  int64_t cta_end = cta_begin + units_per_cta;
+  if (cta_end > n_units) cta_end = n_units;
+  bool bad = false;
+  for (int64_t unit = cta_begin + warp; unit < cta_end; unit += SYNC_WARPS) {
+    const int seg = find_seg(segs, n_segs, unit);
+    if (!MULOCO_IN_BOUNDS(seg >= 0 && seg < n_segs, status)) return;
+    const SyncSeg s = segs[seg];
+    if (!MULOCO_IN_BOUNDS(unit - s.unit_begin < s.rows * s.nblk, status)) return;
+    UnitPos u = unit_pos(s, unit, 128, lane);
+    if (u.nvalid == 0) continue;
+    float* r1 = reps[s.rep_index];
+    u.vec = u.vec && ((((uintptr_t)r1) & 15) == 0);
+    float tg[4], r[4], psi[4];
+    load4(s.theta_g + u.off, u.vec, u.nvalid, tg);
+    load4(r1 + u.off, u.vec, u.nvalid, r);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      psi[e] = __fsub_rn(tg[e], r[e]);
+      if (e < u.nvalid && !(fabsf(psi[e]) <= FLT_MAX)) bad = true;
+    }
+    store4(s.u + u.off, u.vec, u.nvalid, psi);
+    store4(s.theta_g + u.off, u.vec, u.nvalid, r);
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, ST_NONFINITE);
+}
+
 }  // namespace
 
 void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas,
@@ -922,6 +958,14 @@ void launch_outer_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* 
     launch_sync_q<2>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
   else
     launch_sync_q<0>(st, grid, segs, n_segs, replicas, K, n_units, upc, block, outer_lr, mu, inv_k, status);
+}
+
+void launch_dp_sync(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int64_t n_units,
+                    int* status) {
+  if (n_units <= 0) return;
+  const int64_t upc = (int64_t)SYNC_WARPS * SYNC_UNITS_PER_WARP;
+  dim3 grid((unsigned)((n_units + upc - 1) / upc));
+  dp_sync_kernel<<<grid, SYNC_THREADS, 0, st>>>(segs, n_segs, replicas, n_units, upc, status);
 }
 
 void launch_shard_delta(cudaStream_t st, const SyncSeg* segs, int n_segs, float* const* replicas, int K,
