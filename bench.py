@@ -602,7 +602,8 @@ def run_e2e(opt, w, torch, dist, world):
     elt = 2 if w.grad_dtype == "bf16" else 4
     set_bytes = opt.flat_numel * elt
     avail = psutil.virtual_memory().available
-    n_sets = w.K if set_bytes * w.K * 1.5 < avail else 1
+    # every rank of the node pins its own sets: share the host memory that is free now
+    n_sets = w.K if set_bytes * w.K * 1.5 < avail / max(world, 1) else 1
     # drop the device-resident gradients: in this mode they come from the host each step
     opt.grads = None; opt.flat_grads = None; opt._grad_table_all = None
     torch.cuda.empty_cache()
