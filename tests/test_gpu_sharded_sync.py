@@ -164,3 +164,33 @@ def test_sharded_sync_argument_errors(nccl_one_rank):
     with pytest.raises(binding.MulocoError):
         g.shard_layout(-1, 2, 2)                               # rank outside the world
     g.close()
+
+
+def test_config1_full_size_sharded_sync_equals_the_fused_sync(nccl_one_rank):
+    """The benchmark's 150M-shaped workload at full size (8 replicas of 134M parameters, two
+    inner steps with the benchmark's gradient recipe, then the sync): the three-pass path over a
+    one-rank NCCL communicator must leave theta, u and every replica bit-equal to the fused kernel."""
+    import torch
+    from paper_2505_23725_b200 import binding
+    w = configs.workload(1)
+    outs = []
+    for sharded in (False, True):
+        opt = binding.MuLoCo(w, "cuda:0", init_seed=11, alloc_grads=True)
+        for step in range(2):
+            synth.torch_fill_gradients(opt.grads, w.tensors, w.K, 100 + step, opt.device)
+            opt.inner_step(-1, None, 1.0)
+        if sharded:
+            assert opt.sharded_outer_sync(-1, nccl_one_rank) == 0      # one rank: nothing on the wire
+        else:
+            opt.outer_sync(-1)
+        opt.sync_status()
+        # per tensor (the flat buffers have uninitialised padding between tensors)
+        outs.append([(opt.theta_g[i].clone(), opt.outer_u[i].clone(), opt.theta_k[0][i].clone(),
+                      opt.theta_k[w.K - 1][i].clone()) for i in range(opt.n)])
+        opt.close()
+        del opt
+        torch.cuda.empty_cache()
+    for i, (fused, shard) in enumerate(zip(outs[0], outs[1])):
+        for a, b, what in zip(fused, shard, ("theta", "u", "replica 0", "replica K-1")):
+            assert torch.equal(a, b), f"tensor {i}: {what}"
+        assert torch.equal(shard[2], shard[0]) and torch.equal(shard[3], shard[0])
